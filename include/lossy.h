@@ -1,0 +1,217 @@
+/*
+ * lossy.h — C ABI of the packet-loss-tolerant data-parallel step for one B200.
+ *
+ * The library simulates, inside one GPU's HBM, the iteration of the paper's
+ * "Model Formulation" section for W workers that each own one shard of a flat
+ * parameter bucket:
+ *
+ *   (2) gradient communication  -> lossy_aggregate   (unbiased estimate, Section 3 step (2))
+ *   (3) local update            -> lossy_step        (Section 3 step (3); SGD or Adam)
+ *   (4) parameter broadcast     -> lossy_broadcast   (Section 3 step (4), stale retention)
+ *   drift between replicas      -> drift_norms       ("Quantifying Model Drift")
+ *   all four in one pass        -> lossy_fused_step
+ *
+ * Conventions shared by every entry point
+ *   - Every data pointer is DEVICE memory owned by the caller unless the comment
+ *     says "host". Pointer tables (`grads`, `replicas`) are HOST arrays of W
+ *     device pointers; they are copied into the kernel arguments at the call.
+ *   - All data pointers must be 16-byte aligned. `packet_elems` must be a
+ *     multiple of 8 so that every packet starts on a 16-byte boundary in both
+ *     supported element types.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream). Calls are asynchronous on that stream and never synchronise.
+ *   - `step` is 1-based: it is the hash's step counter and Adam's t.
+ *   - Return value: LOSSY_OK or an error code; nothing throws, nothing traps on
+ *     the device. A bad argument is rejected before any launch.
+ *   - The bucket is cut into K = ceil(n / packet_elems) packets of
+ *     `packet_elems` contiguous elements (the last may be short). Shard j, owned
+ *     by worker j, is the contiguous packet range [j*pps, min(K,(j+1)*pps)) with
+ *     pps = ceil(K / W)  (Section 3: theta = (theta^(1) ... theta^(N))).
+ *   - Packet k of the bucket has the global packet id packet_base + k; only the
+ *     drop-mask hash sees the global id, so a model can be streamed bucket by
+ *     bucket with independent masks.
+ */
+#ifndef LOSSY_H_
+#define LOSSY_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lossy_ctx lossy_ctx; /* opaque; host object + small device scratch */
+
+enum { LOSSY_OK = 0, LOSSY_EINVAL = 1, LOSSY_ENOMEM = 2, LOSSY_ECUDA = 3 };
+enum { LOSSY_F32 = 0, LOSSY_BF16 = 1 };  /* element types of gradients / replicas */
+enum { LOSSY_SGD = 0, LOSSY_ADAM = 1 };
+enum {
+  /* The owner's own gradient piece (src == dst) is always delivered. Default (flag
+   * clear) follows the estimator as printed: the sum runs over all N workers and
+   * every indicator is Bernoulli(1-p). */
+  LOSSY_SELF_LOSSLESS = 1u,
+  /* A packet that received nothing leaves theta, m, v untouched. Default: the
+   * estimate is exactly 0 and is fed to the unmodified optimizer. */
+  LOSSY_ZERO_SKIP = 2u
+};
+
+#define LOSSY_MAX_WORKERS 64u
+
+typedef struct {
+  uint32_t W;            /* workers = shards = replicas, 1..64 (the paper's N)           */
+  uint32_t packet_elems; /* P > 0, multiple of 8                                        */
+  uint64_t n;            /* elements in the bucket; 0 makes every call a no-op          */
+  uint64_t packet_base;  /* global id of this bucket's packet 0                         */
+  double   p_grad;       /* drop probability of a gradient packet, in [0,1)             */
+  double   p_param;      /* drop probability of a broadcast packet, in [0,1)            */
+  uint64_t seed;         /* hash key; same seed => same masks, on host and device       */
+  uint32_t grad_dtype;   /* LOSSY_F32 or LOSSY_BF16                                     */
+  uint32_t replica_dtype;/* LOSSY_F32 or LOSSY_BF16 (bf16 = round-to-nearest-even cast) */
+  uint32_t optimizer;    /* LOSSY_SGD or LOSSY_ADAM                                     */
+  uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP                  */
+  float lr, beta1, beta2, eps; /* eta_t and Adam's constants (beta/eps unused for SGD)  */
+} lossy_config;
+
+/*
+ * lossy_init — validate `cfg`, derive the integer drop thresholds
+ * T = floor(p * 2^32) (a packet is dropped iff its 32-bit hash value is < T, so
+ * p = 0 never drops) and allocate the per-block partial sums the drift reduction
+ * needs on the CURRENT device. `*out` receives the context; free it with
+ * lossy_destroy. Section 3 fixes W (= N), p; Algorithm 1 separates p_grad and
+ * p_param; Theorem "Bounded Model Drift" requires p < 1.
+ * Errors: LOSSY_EINVAL (W = 0 or > 64, P = 0 or not a multiple of 8, p outside
+ * [0,1), unknown enum, NULL pointer), LOSSY_ENOMEM, LOSSY_ECUDA.
+ */
+int lossy_init(const lossy_config* cfg, lossy_ctx** out);
+
+/* lossy_destroy — free the context and its device scratch. NULL is allowed. */
+void lossy_destroy(lossy_ctx* ctx);
+
+/*
+ * lossy_set_lr — change eta_t for the following steps (Section 3 step (3) lets the
+ * learning rate depend on t). Returns LOSSY_EINVAL for a NULL context.
+ */
+int lossy_set_lr(lossy_ctx* ctx, float lr);
+
+/*
+ * lossy_aggregate — Section 3 step (2) and "Unbiased Gradient Aggregation":
+ * for every packet k with owner j,
+ *     s_i   = 1 iff hash(seed, step, src=i, dst=j, packet_base+k) >= T_grad
+ *     c_k   = sum_i s_i
+ *     ghat[e] = (sum over i ascending with s_i = 1 of float(g_i[e])) / float(c_k),  e in packet k
+ *     ghat[e] = 0 when c_k = 0 (the regularised fallback).
+ * The sum is accumulated in fp32 in ascending worker order; the division is an
+ * IEEE fp32 division. Dropped packets are never read.
+ *   grads      host array of W device pointers, each [n] of cfg.grad_dtype (read only)
+ *   ghat       [n] fp32, written
+ *   count      [K] uint8, written (c_k), or NULL
+ *   recv_bits  [K] uint64, written (bit i = s_i), or NULL
+ */
+int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads,
+                    float* ghat, uint8_t* count, uint64_t* recv_bits, void* stream);
+
+/*
+ * lossy_step — Section 3 step (3): the owner's update of its shard with ghat,
+ * in fp32, every operation rounded separately (no fused multiply-add):
+ *   SGD : theta = theta - (lr * ghat)
+ *   Adam: m = b1*m + (1-b1)*ghat;  v = b2*v + ((1-b2)*ghat)*ghat
+ *         theta = theta - (lr * (m*ibc1)) / (sqrt(v*ibc2) + eps)
+ *         ibc1 = float(1/(1-b1^step)), ibc2 = float(1/(1-b2^step)) from double on the host.
+ *   count      [K] uint8 from lossy_aggregate; needed (non-NULL) only with
+ *              LOSSY_ZERO_SKIP, where packets with count 0 are left untouched
+ *   master     [n] fp32, updated in place;  m, v: [n] fp32 (Adam only, else NULL)
+ */
+int lossy_step(lossy_ctx* ctx, uint64_t step, const float* ghat, const uint8_t* count,
+               float* master, float* m, float* v, void* stream);
+
+/*
+ * lossy_broadcast — Section 3 step (4): x = cast(master) is offered to every
+ * replica; replica i takes packet k iff i is its owner or
+ *     hash(seed, step, src=owner, dst=i, packet_base+k) >= T_param,
+ * otherwise the replica's packet is left exactly as it was (stale).
+ *   master     [n] fp32 (read only)
+ *   replicas   host array of W device pointers, each [n] of cfg.replica_dtype
+ *   stale_bits [K] uint64, written (bit i = replica i kept its old packet), or NULL
+ */
+int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master,
+                    void* const* replicas, uint64_t* stale_bits, void* stream);
+
+/*
+ * drift_norms — "Quantifying Model Drift": for every replica i
+ *     d_i = sqrt( sum_e ( float(replica_i[e]) - float(cast(master[e])) )^2 )
+ * i.e. the distance of worker i's copy from the owners' current values.
+ *   norms  [W] fp32, written, or NULL
+ *   sumsq  [W] fp64, the squared sums are ADDED to it (sum several buckets by
+ *          zeroing it once and calling per bucket), or NULL
+ * The reduction order is fixed, so the result is reproducible run to run.
+ */
+int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas,
+                float* norms, double* sumsq, void* stream);
+
+/*
+ * lossy_fused_step — steps (2), (3), (4) and the drift norms in ONE pass over
+ * the bucket; ghat is not materialised unless asked for. The state it leaves
+ * (master, m, v, replicas) and every optional output are bit-identical to the
+ * sequence lossy_aggregate -> lossy_step -> lossy_broadcast -> drift_norms.
+ * Optional outputs (NULL to skip): ghat [n], count [K], recv_bits [K],
+ * stale_bits [K], norms [W], sumsq [W] (added to, as in drift_norms).
+ */
+int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads,
+                     float* master, float* m, float* v, void* const* replicas,
+                     float* ghat, uint8_t* count, uint64_t* recv_bits,
+                     uint64_t* stale_bits, float* norms, double* sumsq, void* stream);
+
+/*
+ * lossy_fused_step_host — the same step for a caller whose gradients live in
+ * HOST memory (pinned memory for full copy speed): copies worker i's gradient
+ * from host_grads[i] into dev_grads[i] on `stream`, runs lossy_fused_step, and
+ * copies the W norms to `host_norms`. It returns after the stream has been
+ * synchronised, so `host_norms` is valid on return.
+ *   host_grads  host array of W HOST pointers, each [n] of cfg.grad_dtype
+ *   dev_grads   host array of W DEVICE staging pointers, each [n], caller-owned
+ *   dev_norms   [W] fp32 device; host_norms [W] fp32 host
+ */
+int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host_grads,
+                          void* const* dev_grads, float* master, float* m, float* v,
+                          void* const* replicas, float* dev_norms, float* host_norms,
+                          void* stream);
+
+/*
+ * lossy_mask — host evaluation of one delivery indicator of Section 3:
+ * returns 1 if the transmission (src -> dst) of global packet `packet` at `step`
+ * is delivered, 0 if dropped, using T_param when `is_param` is non-zero and
+ * T_grad otherwise. The device kernels evaluate the same integer function.
+ * Returns -1 for a NULL context.
+ */
+int lossy_mask(const lossy_ctx* ctx, uint64_t step, uint32_t src, uint32_t dst,
+               uint64_t packet, int is_param);
+
+/*
+ * lossy_hash_u32 — the 32-bit uniform value behind lossy_mask (context-free).
+ */
+uint32_t lossy_hash_u32(uint64_t seed, uint64_t step, uint32_t src, uint32_t dst,
+                        uint64_t packet);
+
+/*
+ * lossy_mask_grid — evaluate delivery indicators on the DEVICE for a dense grid
+ * (a test hook that proves host and device agree): for q in [0, count),
+ * out[q] = delivered(step, src[q], dst[q], packet[q]) as uint8.
+ *   src, dst  [count] uint32 device; packet [count] uint64 device; out [count] uint8 device
+ */
+int lossy_mask_grid(lossy_ctx* ctx, uint64_t step, const uint32_t* src, const uint32_t* dst,
+                    const uint64_t* packet, uint64_t count, int is_param, uint8_t* out,
+                    void* stream);
+
+/* lossy_last_error — text of the last error on this context (host string, never NULL). */
+const char* lossy_last_error(const lossy_ctx* ctx);
+
+/* lossy_num_packets — K = ceil(n / packet_elems) for this context (0 for NULL). */
+uint64_t lossy_num_packets(const lossy_ctx* ctx);
+
+/* lossy_kernel_launches — kernels this context has launched so far (0 for NULL). */
+uint64_t lossy_kernel_launches(const lossy_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOSSY_H_ */
