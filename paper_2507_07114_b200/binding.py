@@ -1,0 +1,196 @@
+"""Thin ctypes binding of the C ABI in include/lossy.h (argument marshalling only).
+
+Every function has the name of the C entry point it calls; tensors are passed as
+raw device pointers and the current torch CUDA stream as the stream argument. All
+arithmetic runs in the CUDA library. There is no fallback: if the shared library
+is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA = 0, 1, 2, 3
+LOSSY_F32, LOSSY_BF16 = 0, 1
+LOSSY_SGD, LOSSY_ADAM = 0, 1
+LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP = 1, 2
+
+EXPORTS = [
+    "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_aggregate", "lossy_step", "lossy_broadcast",
+    "drift_norms", "lossy_fused_step", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
+    "lossy_mask_grid", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
+]
+
+
+class lossy_config(C.Structure):
+    _fields_ = [
+        ("W", C.c_uint32), ("packet_elems", C.c_uint32), ("n", C.c_uint64), ("packet_base", C.c_uint64),
+        ("p_grad", C.c_double), ("p_param", C.c_double), ("seed", C.c_uint64),
+        ("grad_dtype", C.c_uint32), ("replica_dtype", C.c_uint32), ("optimizer", C.c_uint32),
+        ("flags", C.c_uint32), ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
+        ("eps", C.c_float),
+    ]
+
+
+class LossyError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"lossy error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> C.CDLL:
+    """dlopen liblossy_b200.so (built in-tree by paper_2507_07114_b200.build) and declare its signatures."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or _build.LIB_PATH
+    if not os.path.exists(path):
+        raise FileNotFoundError(f"{path} is missing: run paper_2507_07114_b200.build.build() (needs nvcc); "
+                                "there is no CPU fallback")
+    lib = C.CDLL(path)
+    vp, u64, u32 = C.c_void_p, C.c_uint64, C.c_uint32
+    lib.lossy_init.restype = C.c_int
+    lib.lossy_init.argtypes = [C.POINTER(lossy_config), C.POINTER(vp)]
+    lib.lossy_destroy.restype = None
+    lib.lossy_destroy.argtypes = [vp]
+    lib.lossy_set_lr.restype = C.c_int
+    lib.lossy_set_lr.argtypes = [vp, C.c_float]
+    lib.lossy_aggregate.restype = C.c_int
+    lib.lossy_aggregate.argtypes = [vp, u64, vp, vp, vp, vp, vp]
+    lib.lossy_step.restype = C.c_int
+    lib.lossy_step.argtypes = [vp, u64, vp, vp, vp, vp, vp, vp]
+    lib.lossy_broadcast.restype = C.c_int
+    lib.lossy_broadcast.argtypes = [vp, u64, vp, vp, vp, vp]
+    lib.drift_norms.restype = C.c_int
+    lib.drift_norms.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.lossy_fused_step.restype = C.c_int
+    lib.lossy_fused_step.argtypes = [vp, u64] + [vp] * 12
+    lib.lossy_fused_step_host.restype = C.c_int
+    lib.lossy_fused_step_host.argtypes = [vp, u64] + [vp] * 9
+    lib.lossy_mask.restype = C.c_int
+    lib.lossy_mask.argtypes = [vp, u64, u32, u32, u64, C.c_int]
+    lib.lossy_hash_u32.restype = u32
+    lib.lossy_hash_u32.argtypes = [u64, u64, u32, u32, u64]
+    lib.lossy_mask_grid.restype = C.c_int
+    lib.lossy_mask_grid.argtypes = [vp, u64, vp, vp, vp, u64, C.c_int, vp, vp]
+    lib.lossy_last_error.restype = C.c_char_p
+    lib.lossy_last_error.argtypes = [vp]
+    lib.lossy_num_packets.restype = u64
+    lib.lossy_num_packets.argtypes = [vp]
+    lib.lossy_kernel_launches.restype = u64
+    lib.lossy_kernel_launches.argtypes = [vp]
+    if path == _build.LIB_PATH:
+        _lib = lib
+    return lib
+
+
+def _dt(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return LOSSY_F32
+    if t == torch.bfloat16:
+        return LOSSY_BF16
+    raise TypeError(f"unsupported element type {t}")
+
+
+def _p(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _table(ts):
+    return (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(ctx, rc):
+    if rc != LOSSY_OK:
+        raise LossyError(rc, load_library().lossy_last_error(ctx).decode())
+
+
+def lossy_init(*, W, n, packet_elems, p_grad, p_param, seed, grad_dtype, replica_dtype, optimizer, lr,
+               beta1=0.9, beta2=0.95, eps=1e-8, flags=0, packet_base=0):
+    """Create a context on the current CUDA device; returns an opaque handle (free with lossy_destroy)."""
+    lib = load_library()
+    torch.cuda.init()
+    opt = {"sgd": LOSSY_SGD, "adam": LOSSY_ADAM}.get(optimizer, optimizer)
+    cfg = lossy_config(W, packet_elems, n, packet_base, p_grad, p_param, seed, _dt(grad_dtype), _dt(replica_dtype),
+                       opt, flags, lr, beta1, beta2, eps)
+    ctx = C.c_void_p()
+    with torch.cuda.device(torch.cuda.current_device()):
+        rc = lib.lossy_init(C.byref(cfg), C.byref(ctx))
+    if rc != LOSSY_OK:
+        raise LossyError(rc, "lossy_init rejected the configuration" if rc == LOSSY_EINVAL else "lossy_init failed")
+    return ctx
+
+
+def lossy_destroy(ctx):
+    load_library().lossy_destroy(ctx)
+
+
+def lossy_set_lr(ctx, lr):
+    _check(ctx, load_library().lossy_set_lr(ctx, lr))
+
+
+def lossy_aggregate(ctx, step, grads, ghat, count=None, recv_bits=None):
+    _check(ctx, load_library().lossy_aggregate(ctx, step, _table(grads), _p(ghat), _p(count), _p(recv_bits),
+                                               _stream()))
+
+
+def lossy_step(ctx, step, ghat, count, master, m=None, v=None):
+    _check(ctx, load_library().lossy_step(ctx, step, _p(ghat), _p(count), _p(master), _p(m), _p(v), _stream()))
+
+
+def lossy_broadcast(ctx, step, master, replicas, stale_bits=None):
+    _check(ctx, load_library().lossy_broadcast(ctx, step, _p(master), _table(replicas), _p(stale_bits), _stream()))
+
+
+def drift_norms(ctx, master, replicas, norms=None, sumsq=None):
+    _check(ctx, load_library().drift_norms(ctx, _p(master), _table(replicas), _p(norms), _p(sumsq), _stream()))
+
+
+def lossy_fused_step(ctx, step, grads, master, m, v, replicas, ghat=None, count=None, recv_bits=None,
+                     stale_bits=None, norms=None, sumsq=None):
+    _check(ctx, load_library().lossy_fused_step(ctx, step, _table(grads), _p(master), _p(m), _p(v), _table(replicas),
+                                                _p(ghat), _p(count), _p(recv_bits), _p(stale_bits), _p(norms),
+                                                _p(sumsq), _stream()))
+
+
+def lossy_fused_step_host(ctx, step, host_grads, dev_grads, master, m, v, replicas, dev_norms, host_norms):
+    """host_grads: W pinned CPU tensors; host_norms: a CPU fp32 tensor of W elements (valid on return)."""
+    _check(ctx, load_library().lossy_fused_step_host(ctx, step, _table(host_grads), _table(dev_grads), _p(master),
+                                                     _p(m), _p(v), _table(replicas), _p(dev_norms), _p(host_norms),
+                                                     _stream()))
+
+
+def lossy_mask(ctx, step, src, dst, packet, is_param=False) -> int:
+    return load_library().lossy_mask(ctx, step, src, dst, packet, int(is_param))
+
+
+def lossy_hash_u32(seed, step, src, dst, packet) -> int:
+    return load_library().lossy_hash_u32(seed, step, src, dst, packet)
+
+
+def lossy_mask_grid(ctx, step, src, dst, packet, out, is_param=False):
+    _check(ctx, load_library().lossy_mask_grid(ctx, step, _p(src), _p(dst), _p(packet), src.numel(), int(is_param),
+                                               _p(out), _stream()))
+
+
+def lossy_last_error(ctx) -> str:
+    return load_library().lossy_last_error(ctx).decode()
+
+
+def lossy_num_packets(ctx) -> int:
+    return load_library().lossy_num_packets(ctx)
+
+
+def lossy_kernel_launches(ctx) -> int:
+    return load_library().lossy_kernel_launches(ctx)

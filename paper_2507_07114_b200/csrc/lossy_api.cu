@@ -1,0 +1,338 @@
+// C ABI of the lossy data-parallel step (see include/lossy.h for the contract).
+// Host side: argument validation, threshold and hash-key derivation, launches.
+#include "../../include/lossy.h"
+
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "lossy_kernels.cuh"
+
+using namespace lossy;
+
+struct lossy_ctx {
+  lossy_config cfg;
+  uint64_t K;
+  uint32_t chunks_per_packet;
+  uint32_t num_chunks;
+  uint32_t pps;
+  uint32_t Tg, Tp;
+  int device;
+  int num_sms;
+  uint32_t max_blocks;   // capacity of `partials`
+  double* partials;      // device, [max_blocks][kMaxW]
+  uint64_t launches;
+  char err[256];
+};
+
+namespace {
+
+constexpr int kBlocksPerSmCap = 8;
+
+int fail(lossy_ctx* ctx, int code, const char* msg) {
+  if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s", msg);
+  return code;
+}
+int fail_cuda(lossy_ctx* ctx, const char* what, cudaError_t e) {
+  if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s: %s", what, cudaGetErrorString(e));
+  return LOSSY_ECUDA;
+}
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+uint32_t threshold_of(double p) { return (uint32_t)floor(p * 4294967296.0); }
+
+int check_table(lossy_ctx* ctx, const void* const* tab, const char* name) {
+  if (!tab) return fail(ctx, LOSSY_EINVAL, name);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i)
+    if (!tab[i] || !aligned16(tab[i])) return fail(ctx, LOSSY_EINVAL, name);
+  return LOSSY_OK;
+}
+
+void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
+  memset(&P, 0, sizeof P);
+  const lossy_config& c = ctx->cfg;
+  P.n = c.n;
+  P.packet_base = c.packet_base;
+  P.step_key = step_key_of(c.seed, step);
+  P.num_chunks = ctx->num_chunks;
+  P.chunks_per_packet = ctx->chunks_per_packet;
+  P.pps = ctx->pps;
+  P.P = c.packet_elems;
+  P.W = c.W;
+  P.Tg = ctx->Tg;
+  P.Tp = ctx->Tp;
+  P.flags = c.flags;
+  P.lr = c.lr;
+  P.b1 = c.beta1;
+  P.b2 = c.beta2;
+  P.omb1 = 1.0f - c.beta1;   // (1 - beta) in fp32
+  P.omb2 = 1.0f - c.beta2;
+  P.ibc1 = (float)(1.0 / (1.0 - pow((double)c.beta1, (double)step)));
+  P.ibc2 = (float)(1.0 / (1.0 - pow((double)c.beta2, (double)step)));
+  P.eps = c.eps;
+  P.partials = ctx->partials;
+}
+
+template <int PH, class GT, class RT, int OPT>
+int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out) {
+  auto kern = lossy_kernel<PH, GT, RT, OPT>;
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, 0);
+  if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
+  if (per_sm < 1) per_sm = 1;
+  if (per_sm > kBlocksPerSmCap) per_sm = kBlocksPerSmCap;
+  uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
+  const uint32_t need = (P.num_chunks + kWarps - 1) / kWarps;
+  if (blocks > need) blocks = need;
+  if (blocks > ctx->max_blocks) blocks = ctx->max_blocks;
+  if (blocks == 0) blocks = 1;
+  kern<<<blocks, kThreads, 0, s>>>(P);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "kernel launch", e);
+  ctx->launches++;
+  if (blocks_out) *blocks_out = blocks;
+  return LOSSY_OK;
+}
+
+int finalize_drift(lossy_ctx* ctx, uint32_t blocks, float* norms, double* sumsq, cudaStream_t s) {
+  drift_finalize_kernel<<<1, kMaxW, 0, s>>>(ctx->partials, blocks, ctx->cfg.W, norms, sumsq);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "drift finalize launch", e);
+  ctx->launches++;
+  return LOSSY_OK;
+}
+
+// dispatch on the runtime element types / optimizer
+template <int PH>
+int dispatch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks) {
+  const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
+  const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
+  const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
+  if constexpr (PH == AGG) {
+    return gb ? launch<PH, BF16, F32, 0>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
+  } else if constexpr (PH == STEP) {
+    return adam ? launch<PH, F32, F32, 1>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
+  } else if constexpr (PH == BCAST || PH == DRIFT) {
+    return rb ? launch<PH, F32, BF16, 0>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
+  } else {
+    if (gb && rb) return adam ? launch<PH, BF16, BF16, 1>(ctx, P, s, blocks) : launch<PH, BF16, BF16, 0>(ctx, P, s, blocks);
+    if (gb && !rb) return adam ? launch<PH, BF16, F32, 1>(ctx, P, s, blocks) : launch<PH, BF16, F32, 0>(ctx, P, s, blocks);
+    if (!gb && rb) return adam ? launch<PH, F32, BF16, 1>(ctx, P, s, blocks) : launch<PH, F32, BF16, 0>(ctx, P, s, blocks);
+    return adam ? launch<PH, F32, F32, 1>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
+  if (!cfg || !out) return LOSSY_EINVAL;
+  *out = nullptr;
+  if (cfg->W == 0 || cfg->W > LOSSY_MAX_WORKERS) return LOSSY_EINVAL;
+  if (cfg->packet_elems == 0 || cfg->packet_elems % 8 != 0) return LOSSY_EINVAL;
+  if (!(cfg->p_grad >= 0.0 && cfg->p_grad < 1.0) || !(cfg->p_param >= 0.0 && cfg->p_param < 1.0)) return LOSSY_EINVAL;
+  if (cfg->grad_dtype > LOSSY_BF16 || cfg->replica_dtype > LOSSY_BF16 || cfg->optimizer > LOSSY_ADAM) return LOSSY_EINVAL;
+  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP)) return LOSSY_EINVAL;
+  const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
+  const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;
+  if (K * cpp >= (1ull << 31)) return LOSSY_EINVAL;  // stream larger models bucket by bucket
+
+  lossy_ctx* ctx = new (std::nothrow) lossy_ctx;
+  if (!ctx) return LOSSY_ENOMEM;
+  memset(ctx, 0, sizeof *ctx);
+  ctx->cfg = *cfg;
+  ctx->K = K;
+  ctx->chunks_per_packet = (uint32_t)cpp;
+  ctx->num_chunks = (uint32_t)(K * cpp);
+  const uint64_t pps = (K + cfg->W - 1) / cfg->W;
+  ctx->pps = pps ? (uint32_t)pps : 1u;
+  ctx->Tg = threshold_of(cfg->p_grad);
+  ctx->Tp = threshold_of(cfg->p_param);
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  if (e != cudaSuccess) { delete ctx; return LOSSY_ECUDA; }
+  ctx->max_blocks = (uint32_t)(ctx->num_sms * kBlocksPerSmCap);
+  e = cudaMalloc(&ctx->partials, (size_t)ctx->max_blocks * kMaxW * sizeof(double));
+  if (e != cudaSuccess) { delete ctx; return e == cudaErrorMemoryAllocation ? LOSSY_ENOMEM : LOSSY_ECUDA; }
+  *out = ctx;
+  return LOSSY_OK;
+}
+
+void lossy_destroy(lossy_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->partials) cudaFree(ctx->partials);
+  delete ctx;
+}
+
+int lossy_set_lr(lossy_ctx* ctx, float lr) {
+  if (!ctx) return LOSSY_EINVAL;
+  ctx->cfg.lr = lr;
+  return LOSSY_OK;
+}
+
+int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat, uint8_t* count,
+                    uint64_t* recv_bits, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
+  if (!ghat || !aligned16(ghat)) return fail(ctx, LOSSY_EINVAL, "ghat: NULL or misaligned");
+  Params P;
+  fill_common(ctx, step, P);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.grads[i] = grads[i];
+  P.ghat = ghat;
+  P.count = count;
+  P.recv_bits = recv_bits;
+  return dispatch<AGG>(ctx, P, (cudaStream_t)stream, nullptr);
+}
+
+int lossy_step(lossy_ctx* ctx, uint64_t step, const float* ghat, const uint8_t* count, float* master, float* m,
+               float* v, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  if (step == 0) return fail(ctx, LOSSY_EINVAL, "step is 1-based");
+  if (!ghat || !aligned16(ghat) || !master || !aligned16(master)) return fail(ctx, LOSSY_EINVAL, "ghat/master: NULL or misaligned");
+  if (ctx->cfg.optimizer == LOSSY_ADAM && (!m || !v || !aligned16(m) || !aligned16(v)))
+    return fail(ctx, LOSSY_EINVAL, "Adam needs m and v");
+  if ((ctx->cfg.flags & LOSSY_ZERO_SKIP) && !count) return fail(ctx, LOSSY_EINVAL, "LOSSY_ZERO_SKIP needs count");
+  Params P;
+  fill_common(ctx, step, P);
+  P.ghat = const_cast<float*>(ghat);
+  P.count_in = count;
+  P.master = master;
+  P.m = m;
+  P.v = v;
+  return dispatch<STEP>(ctx, P, (cudaStream_t)stream, nullptr);
+}
+
+int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master, void* const* replicas, uint64_t* stale_bits,
+                    void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (!master || !aligned16(master)) return fail(ctx, LOSSY_EINVAL, "master: NULL or misaligned");
+  Params P;
+  fill_common(ctx, step, P);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.replicas[i] = replicas[i];
+  P.master = const_cast<float*>(master);
+  P.stale_bits = stale_bits;
+  return dispatch<BCAST>(ctx, P, (cudaStream_t)stream, nullptr);
+}
+
+int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas, float* norms, double* sumsq,
+                void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (ctx->cfg.n == 0) {
+    if (norms) {
+      cudaError_t e = cudaMemsetAsync(norms, 0, ctx->cfg.W * sizeof(float), (cudaStream_t)stream);
+      if (e != cudaSuccess) return fail_cuda(ctx, "memset", e);
+    }
+    return LOSSY_OK;
+  }
+  if (!master || !aligned16(master)) return fail(ctx, LOSSY_EINVAL, "master: NULL or misaligned");
+  Params P;
+  fill_common(ctx, 1, P);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.replicas[i] = const_cast<void*>(replicas[i]);
+  P.master = const_cast<float*>(master);
+  uint32_t blocks = 0;
+  if (int rc = dispatch<DRIFT>(ctx, P, (cudaStream_t)stream, &blocks)) return rc;
+  return finalize_drift(ctx, blocks, norms, sumsq, (cudaStream_t)stream);
+}
+
+int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* master, float* m, float* v,
+                     void* const* replicas, float* ghat, uint8_t* count, uint64_t* recv_bits, uint64_t* stale_bits,
+                     float* norms, double* sumsq, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (step == 0) return fail(ctx, LOSSY_EINVAL, "step is 1-based");
+  if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
+  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (ctx->cfg.n == 0) {
+    if (norms) {
+      cudaError_t e = cudaMemsetAsync(norms, 0, ctx->cfg.W * sizeof(float), (cudaStream_t)stream);
+      if (e != cudaSuccess) return fail_cuda(ctx, "memset", e);
+    }
+    return LOSSY_OK;
+  }
+  if (!master || !aligned16(master)) return fail(ctx, LOSSY_EINVAL, "master: NULL or misaligned");
+  if (ctx->cfg.optimizer == LOSSY_ADAM && (!m || !v || !aligned16(m) || !aligned16(v)))
+    return fail(ctx, LOSSY_EINVAL, "Adam needs m and v");
+  if (ghat && !aligned16(ghat)) return fail(ctx, LOSSY_EINVAL, "ghat: misaligned");
+  Params P;
+  fill_common(ctx, step, P);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) {
+    P.grads[i] = grads[i];
+    P.replicas[i] = replicas[i];
+  }
+  P.master = master;
+  P.m = m;
+  P.v = v;
+  P.ghat = ghat;
+  P.count = count;
+  P.recv_bits = recv_bits;
+  P.stale_bits = stale_bits;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (norms || sumsq) {
+    uint32_t blocks = 0;
+    if (int rc = dispatch<AGG | STEP | BCAST | DRIFT>(ctx, P, s, &blocks)) return rc;
+    return finalize_drift(ctx, blocks, norms, sumsq, s);
+  }
+  return dispatch<AGG | STEP | BCAST>(ctx, P, s, nullptr);
+}
+
+int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host_grads, void* const* dev_grads,
+                          float* master, float* m, float* v, void* const* replicas, float* dev_norms,
+                          float* host_norms, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (!host_grads || !dev_grads || !dev_norms || !host_norms) return fail(ctx, LOSSY_EINVAL, "NULL argument");
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t gbytes = (size_t)ctx->cfg.n * (ctx->cfg.grad_dtype == LOSSY_BF16 ? 2 : 4);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) {
+    if (!host_grads[i] || !dev_grads[i]) return fail(ctx, LOSSY_EINVAL, "NULL gradient pointer");
+    if (gbytes) {
+      cudaError_t e = cudaMemcpyAsync(dev_grads[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, s);
+      if (e != cudaSuccess) return fail_cuda(ctx, "gradient upload", e);
+    }
+  }
+  if (int rc = lossy_fused_step(ctx, step, dev_grads, master, m, v, replicas, nullptr, nullptr, nullptr, nullptr,
+                                dev_norms, nullptr, stream))
+    return rc;
+  cudaError_t e = cudaMemcpyAsync(host_norms, dev_norms, ctx->cfg.W * sizeof(float), cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return fail_cuda(ctx, "norm download", e);
+  e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(ctx, "stream synchronize", e);
+  return LOSSY_OK;
+}
+
+uint32_t lossy_hash_u32(uint64_t seed, uint64_t step, uint32_t src, uint32_t dst, uint64_t packet) {
+  return pair_hash(packet_key_of(step_key_of(seed, step), packet), src, dst);
+}
+
+int lossy_mask(const lossy_ctx* ctx, uint64_t step, uint32_t src, uint32_t dst, uint64_t packet, int is_param) {
+  if (!ctx) return -1;
+  const uint32_t T = is_param ? ctx->Tp : ctx->Tg;
+  return lossy_hash_u32(ctx->cfg.seed, step, src, dst, packet) >= T ? 1 : 0;
+}
+
+int lossy_mask_grid(lossy_ctx* ctx, uint64_t step, const uint32_t* src, const uint32_t* dst, const uint64_t* packet,
+                    uint64_t count, int is_param, uint8_t* out, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (count == 0) return LOSSY_OK;
+  if (!src || !dst || !packet || !out) return fail(ctx, LOSSY_EINVAL, "NULL argument");
+  const uint64_t blocks = (count + 255) / 256;
+  if (blocks > 0x7FFFFFFFull) return fail(ctx, LOSSY_EINVAL, "grid too large");
+  mask_grid_kernel<<<(uint32_t)blocks, 256, 0, (cudaStream_t)stream>>>(ctx->cfg.seed, step, src, dst, packet, count,
+                                                                      is_param ? ctx->Tp : ctx->Tg, out);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "mask grid launch", e);
+  ctx->launches++;
+  return LOSSY_OK;
+}
+
+const char* lossy_last_error(const lossy_ctx* ctx) { return ctx ? ctx->err : "NULL context"; }
+uint64_t lossy_num_packets(const lossy_ctx* ctx) { return ctx ? ctx->K : 0; }
+uint64_t lossy_kernel_launches(const lossy_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

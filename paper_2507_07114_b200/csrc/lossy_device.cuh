@@ -1,0 +1,173 @@
+// Device-side building blocks of the lossy data-parallel step (sm_100a).
+//
+// Work decomposition shared by every kernel here: the bucket is walked in
+// "chunks" of 256 contiguous elements (one warp, 8 elements = 16 or 32 bytes per
+// lane) that never straddle a packet, so the delivery masks of a chunk are
+// warp-uniform. Chunk q belongs to packet k = q / chunks_per_packet. Warps take
+// chunks grid-stride, so at any moment the grid streams one contiguous window
+// of every buffer.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lossy {
+
+constexpr int kMaxW = 64;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kChunk = 256;  // elements per warp-chunk
+
+enum Phase : int { AGG = 1, STEP = 2, BCAST = 4, DRIFT = 8 };
+
+struct Params {
+  const void* grads[kMaxW];
+  void* replicas[kMaxW];
+  float* master;
+  float* m;
+  float* v;
+  float* ghat;            // AGG: optional output; STEP without AGG: input
+  uint8_t* count;         // optional output (AGG)
+  uint64_t* recv_bits;    // optional output (AGG)
+  uint64_t* stale_bits;   // optional output (BCAST)
+  const uint8_t* count_in;  // STEP without AGG and ZERO_SKIP: received counts
+  double* partials;       // DRIFT: [gridDim.x][kMaxW] per-block squared sums
+  uint64_t n;
+  uint64_t packet_base;
+  uint64_t step_key;      // hash key of (seed, step), derived on the host
+  uint32_t num_chunks;    // K * chunks_per_packet
+  uint32_t chunks_per_packet;
+  uint32_t pps;           // packets per shard
+  uint32_t P;
+  uint32_t W;
+  uint32_t Tg, Tp;        // drop iff hash < T
+  uint32_t flags;
+  float lr, b1, b2, omb1, omb2, ibc1, ibc2, eps;
+};
+
+// ---- delivery-indicator hash (Section 3: s, r ~ Bernoulli(1-p)) -------------
+// 64-bit finalizer of the splitmix64 generator; the constants of the keyed
+// rounds are this library's own choice and are part of its documented contract.
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ULL;
+  z ^= z >> 27; z *= 0x94D049BB133111EBULL;
+  z ^= z >> 31;
+  return z;
+}
+__host__ __device__ __forceinline__ uint64_t step_key_of(uint64_t seed, uint64_t step) {
+  return mix64(mix64(seed ^ 0x6A09E667F3BCC908ULL) + step * 0x9E3779B97F4A7C15ULL);
+}
+__host__ __device__ __forceinline__ uint64_t packet_key_of(uint64_t step_key, uint64_t packet) {
+  return mix64(step_key ^ (packet * 0xD6E8FEB86659FD93ULL));
+}
+__host__ __device__ __forceinline__ uint32_t pair_hash(uint64_t packet_key, uint32_t src, uint32_t dst) {
+  const uint64_t pair = ((uint64_t)src << 32) | (uint64_t)dst;
+  return (uint32_t)(mix64(packet_key + pair * 0xC2B2AE3D27D4EB4FULL) >> 32);
+}
+
+// ---- streaming 128-bit memory operations ------------------------------------
+// Everything on this path is touched exactly once per step, so loads and stores
+// carry the evict-first ("streaming") cache operator.
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+  return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ void st_stream(void* p, uint4 v) {
+  __stcs(reinterpret_cast<uint4*>(p), v);
+}
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
+// ---- element-type adapters ----------------------------------------------------
+struct F32 { using raw = float; static constexpr int kVecs = 2; };       // 8 elements = 2 x 16 B
+struct BF16 { using raw = uint16_t; static constexpr int kVecs = 1; };   // 8 elements = 1 x 16 B
+
+template <class T> struct Vec8 { uint4 q[T::kVecs]; };
+
+template <class T>
+__device__ __forceinline__ Vec8<T> load8(const void* base, uint64_t e) {
+  Vec8<T> r;
+  const typename T::raw* p = reinterpret_cast<const typename T::raw*>(base) + e;
+#pragma unroll
+  for (int i = 0; i < T::kVecs; ++i) r.q[i] = ld_stream(reinterpret_cast<const uint4*>(p) + i);
+  return r;
+}
+// Ragged tail of the bucket: the last vector may hold fewer than 8 elements.
+template <class T>
+__device__ __forceinline__ Vec8<T> load8_tail(const void* base, uint64_t e, int nvalid) {
+  Vec8<T> r;
+  typename T::raw tmp[8];
+  const typename T::raw* p = reinterpret_cast<const typename T::raw*>(base) + e;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tmp[i] = i < nvalid ? p[i] : (typename T::raw)0;
+  if constexpr (T::kVecs == 2) {
+    r.q[0] = make_uint4(__float_as_uint(tmp[0]), __float_as_uint(tmp[1]), __float_as_uint(tmp[2]), __float_as_uint(tmp[3]));
+    r.q[1] = make_uint4(__float_as_uint(tmp[4]), __float_as_uint(tmp[5]), __float_as_uint(tmp[6]), __float_as_uint(tmp[7]));
+  } else {
+    r.q[0] = make_uint4((uint32_t)tmp[0] | ((uint32_t)tmp[1] << 16), (uint32_t)tmp[2] | ((uint32_t)tmp[3] << 16),
+                        (uint32_t)tmp[4] | ((uint32_t)tmp[5] << 16), (uint32_t)tmp[6] | ((uint32_t)tmp[7] << 16));
+  }
+  return r;
+}
+template <class T>
+__device__ __forceinline__ void store8(void* base, uint64_t e, const Vec8<T>& v, int nvalid) {
+  typename T::raw* p = reinterpret_cast<typename T::raw*>(base) + e;
+  if (nvalid == 8) {
+#pragma unroll
+    for (int i = 0; i < T::kVecs; ++i) st_stream(reinterpret_cast<uint4*>(p) + i, v.q[i]);
+  } else {
+    const uint32_t* w = reinterpret_cast<const uint32_t*>(&v.q[0]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (i < nvalid) {
+        if constexpr (T::kVecs == 2) p[i] = __uint_as_float(w[i]);
+        else p[i] = (uint16_t)(w[i >> 1] >> ((i & 1) * 16));
+      }
+    }
+  }
+}
+template <class T>
+__device__ __forceinline__ Vec8<T> load8_any(const void* base, uint64_t e, int nvalid) {
+  return nvalid == 8 ? load8<T>(base, e) : load8_tail<T>(base, e, nvalid);
+}
+
+// widen 8 elements to fp32 (bf16 -> fp32 is a 16-bit shift, exact)
+template <class T>
+__device__ __forceinline__ void widen(const Vec8<T>& v, float (&f)[8]) {
+  const uint32_t* w = reinterpret_cast<const uint32_t*>(&v.q[0]);
+  if constexpr (T::kVecs == 2) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(w[i]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+}
+// narrow 8 fp32 values to the wire type (bf16: IEEE round-to-nearest-even)
+template <class T>
+__device__ __forceinline__ Vec8<T> narrow(const float (&f)[8]) {
+  Vec8<T> r;
+  uint32_t* w = reinterpret_cast<uint32_t*>(&r.q[0]);
+  if constexpr (T::kVecs == 2) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = __float_as_uint(f[i]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  }
+  return r;
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xFFFFFFFFu, x, o));
+  return x;
+}
+
+}  // namespace lossy

@@ -1,0 +1,225 @@
+// The kernels of the lossy data-parallel step: one template, specialised by the
+// phases it runs. Fused = AGG|STEP|BCAST|DRIFT in a single pass over the bucket.
+#pragma once
+#include "lossy_device.cuh"
+
+namespace lossy {
+
+// One optimizer update of 8 elements, every operation rounded on its own
+// (Section 3 step (3); Adam as bias-corrected Kingma-Ba with host-side corrections).
+template <int OPT>
+__device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8], float (&th)[8], float (&m)[8],
+                                           float (&v)[8]) {
+#pragma unroll
+  for (int x = 0; x < 8; ++x) {
+    if constexpr (OPT == 0) {
+      th[x] = __fsub_rn(th[x], __fmul_rn(P.lr, g[x]));
+    } else {
+      const float mn = __fadd_rn(__fmul_rn(P.b1, m[x]), __fmul_rn(P.omb1, g[x]));
+      const float vn = __fadd_rn(__fmul_rn(P.b2, v[x]), __fmul_rn(__fmul_rn(P.omb2, g[x]), g[x]));
+      const float mh = __fmul_rn(mn, P.ibc1);
+      const float vh = __fmul_rn(vn, P.ibc2);
+      const float den = __fadd_rn(__fsqrt_rn(vh), P.eps);
+      th[x] = __fsub_rn(th[x], __fdiv_rn(__fmul_rn(P.lr, mh), den));
+      m[x] = mn;
+      v[x] = vn;
+    }
+  }
+}
+
+template <int PH, class GT, class RT, int OPT>
+__global__ void __launch_bounds__(kThreads) lossy_kernel(const __grid_constant__ Params P) {
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const uint32_t W = P.W;
+
+  // per-lane drift accumulators: lane l holds replicas l and l + 32
+  double dacc0 = 0.0, dacc1 = 0.0;
+
+  const uint32_t warps_in_grid = gridDim.x * kWarps;
+  for (uint32_t q = blockIdx.x * kWarps + warp; q < P.num_chunks; q += warps_in_grid) {
+    const uint32_t k = q / P.chunks_per_packet;
+    const uint32_t c = q - k * P.chunks_per_packet;
+    const uint32_t j = k / P.pps;  // owner W_j of packet k
+    const uint32_t in_pkt = c * kChunk + lane * 8;
+    const uint64_t e = (uint64_t)k * P.P + in_pkt;
+    int nvalid = 0;
+    if (in_pkt < P.P && e < P.n) nvalid = (P.n - e >= 8) ? 8 : (int)(P.n - e);
+
+    // ---- delivery indicators of this packet (warp-uniform) -------------------
+    const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k);
+    uint64_t recv = 0, stale = 0;
+    if constexpr (PH & AGG) {
+      const uint32_t i0 = lane, i1 = lane + 32;
+      bool s0 = i0 < W && (pair_hash(pkey, i0, j) >= P.Tg || ((P.flags & 1u) && i0 == j));
+      uint32_t lo = __ballot_sync(0xFFFFFFFFu, s0), hi = 0;
+      if (W > 32) {
+        bool s1 = i1 < W && (pair_hash(pkey, i1, j) >= P.Tg || ((P.flags & 1u) && i1 == j));
+        hi = __ballot_sync(0xFFFFFFFFu, s1);
+      }
+      recv = ((uint64_t)hi << 32) | lo;
+    }
+    if constexpr (PH & BCAST) {
+      const uint32_t i0 = lane, i1 = lane + 32;
+      bool d0 = i0 < W && i0 != j && pair_hash(pkey, j, i0) < P.Tp;
+      uint32_t lo = __ballot_sync(0xFFFFFFFFu, d0), hi = 0;
+      if (W > 32) {
+        bool d1 = i1 < W && i1 != j && pair_hash(pkey, j, i1) < P.Tp;
+        hi = __ballot_sync(0xFFFFFFFFu, d1);
+      }
+      stale = ((uint64_t)hi << 32) | lo;
+    }
+    uint32_t cnt = __popcll(recv);
+    if (c == 0 && lane == 0) {
+      if constexpr (PH & AGG) {
+        if (P.count) P.count[k] = (uint8_t)cnt;
+        if (P.recv_bits) P.recv_bits[k] = recv;
+      }
+      if constexpr (PH & BCAST) {
+        if (P.stale_bits) P.stale_bits[k] = stale;
+      }
+    }
+    // Lanes past a short packet or past the bucket end keep nvalid == 0: they stay in the
+    // warp for the shuffles below and every load/store helper skips them.
+
+    // stale copies are read late (for the drift term): start them toward L2 now
+    if constexpr ((PH & BCAST) && (PH & DRIFT)) {
+      uint64_t sm = nvalid > 0 ? stale : 0ull;
+      while (sm) {
+        const int i = __ffsll((long long)sm) - 1;
+        sm &= sm - 1;
+        prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e);
+      }
+    }
+
+    // ---- optimizer state: issue these loads before the gradient loop ---------
+    Vec8<F32> rth, rm, rv;
+    if constexpr (PH & (STEP | BCAST | DRIFT)) rth = load8_any<F32>(P.master, e, nvalid);
+    if constexpr ((PH & STEP) && OPT == 1) {
+      rm = load8_any<F32>(P.m, e, nvalid);
+      rv = load8_any<F32>(P.v, e, nvalid);
+    }
+
+    // ---- (2) unbiased aggregate: masked sum in ascending worker order / count --
+    float g[8];
+    if constexpr (PH & AGG) {
+#pragma unroll
+      for (int x = 0; x < 8; ++x) g[x] = 0.0f;
+      for (uint32_t g0 = 0; g0 < W; g0 += 8) {
+        const uint32_t bits = (uint32_t)(recv >> g0) & 0xFFu;
+        if (bits == 0) continue;
+        Vec8<GT> raw[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if ((bits >> u) & 1u) raw[u] = load8_any<GT>(P.grads[g0 + u], e, nvalid);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if ((bits >> u) & 1u) {
+            float f[8];
+            widen<GT>(raw[u], f);
+#pragma unroll
+            for (int x = 0; x < 8; ++x) g[x] = __fadd_rn(g[x], f[x]);
+          }
+      }
+      if (cnt > 0) {
+        const float fc = (float)cnt;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) g[x] = __fdiv_rn(g[x], fc);
+      }
+      if (P.ghat) {
+        Vec8<F32> o = narrow<F32>(g);
+        store8<F32>(P.ghat, e, o, nvalid);
+      }
+    } else if constexpr (PH & STEP) {
+      Vec8<F32> r = load8_any<F32>(P.ghat, e, nvalid);
+      widen<F32>(r, g);
+      cnt = (P.flags & 2u) ? (uint32_t)P.count_in[k] : 1u;
+    }
+
+    // ---- (3) the owner's update ------------------------------------------------
+    float th[8];
+    if constexpr (PH & (STEP | BCAST | DRIFT)) widen<F32>(rth, th);
+    if constexpr (PH & STEP) {
+      if (!((P.flags & 2u) && cnt == 0)) {
+        float m[8], v[8];
+        if constexpr (OPT == 1) {
+          widen<F32>(rm, m);
+          widen<F32>(rv, v);
+        }
+        optimizer8<OPT>(P, g, th, m, v);
+        store8<F32>(P.master, e, narrow<F32>(th), nvalid);
+        if constexpr (OPT == 1) {
+          store8<F32>(P.m, e, narrow<F32>(m), nvalid);
+          store8<F32>(P.v, e, narrow<F32>(v), nvalid);
+        }
+      }
+    }
+
+    // ---- (4) broadcast with stale retention, and the drift of every copy -------
+    if constexpr (PH & (BCAST | DRIFT)) {
+      const Vec8<RT> wire = narrow<RT>(th);
+      float xw[8];
+      widen<RT>(wire, xw);
+      for (uint32_t i = 0; i < W; ++i) {
+        const bool is_stale = (stale >> i) & 1ull;
+        if constexpr (PH & BCAST) {
+          if (!is_stale) {
+            store8<RT>(P.replicas[i], e, wire, nvalid);
+            continue;
+          }
+        }
+        if constexpr (PH & DRIFT) {
+          const Vec8<RT> old = load8_any<RT>(P.replicas[i], e, nvalid);
+          float fo[8];
+          widen<RT>(old, fo);
+          float s = 0.0f;
+#pragma unroll
+          for (int x = 0; x < 8; ++x) {
+            const float d = x < nvalid ? __fsub_rn(fo[x], xw[x]) : 0.0f;
+            s = __fadd_rn(s, __fmul_rn(d, d));
+          }
+          const float tot = warp_sum(s);
+          if ((i & 31u) == (uint32_t)lane) {
+            if (i < 32) dacc0 += (double)tot; else dacc1 += (double)tot;
+          }
+        }
+      }
+    }
+  }
+
+  // ---- per-block drift partials, fixed order ------------------------------------
+  if constexpr (PH & DRIFT) {
+    __shared__ double sh[kWarps][kMaxW];
+    sh[warp][lane] = dacc0;
+    sh[warp][lane + 32] = dacc1;
+    __syncthreads();
+    if (threadIdx.x < kMaxW) {
+      double t = 0.0;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) t += sh[w][threadIdx.x];
+      P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
+    }
+  }
+}
+
+// Sum the per-block partials in block order; add to sumsq, write the norms.
+__global__ void drift_finalize_kernel(const double* __restrict__ partials, uint32_t nblocks, uint32_t W,
+                                      float* norms, double* sumsq) {
+  const uint32_t i = threadIdx.x;
+  if (i >= W) return;
+  double t = 0.0;
+  for (uint32_t b = 0; b < nblocks; ++b) t += partials[(size_t)b * kMaxW + i];
+  if (sumsq) sumsq[i] += t;
+  if (norms) norms[i] = (float)sqrt(t);
+}
+
+// Delivery indicators on a dense grid of tuples (host/device agreement check).
+__global__ void mask_grid_kernel(uint64_t seed, uint64_t step, const uint32_t* src, const uint32_t* dst,
+                                 const uint64_t* packet, uint64_t count, uint32_t T, uint8_t* out) {
+  const uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= count) return;
+  const uint64_t pkey = packet_key_of(step_key_of(seed, step), packet[q]);
+  out[q] = pair_hash(pkey, src[q], dst[q]) >= T ? 1 : 0;
+}
+
+}  // namespace lossy

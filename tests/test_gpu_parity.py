@@ -1,0 +1,185 @@
+"""Element-by-element parity of the CUDA path against the CPU oracle on small and ragged cases."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2507_07114_b200 as L
+import workload
+from parity_util import (GpuRun, assert_rel, assert_same, compare_outputs, compare_state, make_oracle,
+                         run_parity, to_np)
+
+pytestmark = pytest.mark.gpu
+CFG = workload.baseline_workloads()
+LOSSLESS, SKIP = L.LOSSY_SELF_LOSSLESS, L.LOSSY_ZERO_SKIP
+
+
+def test_config1_w4_sgd_fp32_all_steps():
+    w = CFG["cfg1_w4_sgd_f32"]
+    run_parity(w, w.steps)
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_config2_shape_scaled_ragged(fused):
+    # W=8, bf16 grads, Adam, P=2048: 37 packets + a short one whose length is not a multiple of 8
+    w = workload.scaled(CFG["cfg2_w8_layer_adam"], 2048 * 37 + 1003)
+    run_parity(w, 12, fused=fused)
+
+
+@pytest.mark.parametrize("name", ["cfg3_w64_layer_p01", "cfg3_w64_layer_p10"])
+def test_config3_shape_scaled(name):
+    w = workload.scaled(CFG[name], 4096 * 130 + 40)
+    run_parity(w, 6)
+
+
+@pytest.mark.parametrize("P", [256, 1024, 2048, 4096])
+@pytest.mark.parametrize("p", [0.0, 0.01, 0.05, 0.1, 0.3])
+def test_config5_sweep_scaled(P, p):
+    w = workload.scaled(CFG["cfg5_w16_layer_sweep"], 4096 * 40 + 256 * 3, packet_elems=P, p=p)
+    gpu, orc = run_parity(w, 4)
+    if p == 0.0:
+        assert float(gpu.norms.abs().max()) == 0.0
+        assert int(gpu.count.min()) == 16
+
+
+def test_config4_buckets_streamed_with_packet_base():
+    """Bucket-by-bucket streaming: every bucket has its own context, shard map and global packet ids."""
+    base = CFG["cfg4_w8_full_model"]
+    sizes = [2048 * 21, 2048 * 21, 2048 * 13 + 512]
+    pb = 0
+    tot_g, tot_o = np.zeros(8), np.zeros(8)
+    for b, n in enumerate(sizes):
+        w = workload.scaled(base, n, packet_base=pb, seed=100 + b, name=f"cfg4_bucket{b}")
+        gpu, orc = run_parity(w, 3)
+        tot_g += to_np(gpu.sumsq)
+        tot_o += orc.drift_sumsq()
+        pb += w.K
+    assert_rel(np.sqrt(tot_g), np.sqrt(tot_o), "model-level drift norms")
+    # masks depend on the global packet id: the same bucket at another base gives other masks
+    w0 = workload.scaled(base, sizes[0], packet_base=0, seed=100)
+    w1 = workload.scaled(base, sizes[0], packet_base=5, seed=100)
+    g0, _ = run_parity(w0, 1)
+    g1, _ = run_parity(w1, 1)
+    assert not torch.equal(g0.recv, g1.recv)
+
+
+EDGE = [
+    # name, W, n, P, p, opt, gd, rd, flags
+    ("one_worker", 1, 5000, 256, 0.3, "adam", "bf16", "bf16", 0),
+    ("w63", 63, 8 * 700 + 3, 8, 0.2, "sgd", "f32", "f32", 0),
+    ("w33", 33, 264 * 50, 264, 0.1, "adam", "bf16", "f32", 0),
+    ("fewer_packets_than_workers", 8, 3 * 512 - 100, 512, 0.2, "adam", "f32", "bf16", 0),
+    ("single_short_packet", 4, 5, 1024, 0.3, "sgd", "bf16", "bf16", 0),
+    ("tiny_packets", 4, 8 * 1000 + 1, 8, 0.1, "sgd", "bf16", "bf16", 0),
+    ("heavy_loss_zero_received", 3, 64 * 300, 64, 0.7, "adam", "bf16", "bf16", 0),
+    ("heavy_loss_zero_skip", 3, 64 * 300, 64, 0.7, "adam", "bf16", "bf16", SKIP),
+    ("self_lossless", 8, 2048 * 9 + 16, 2048, 0.4, "adam", "bf16", "bf16", LOSSLESS),
+    ("both_flags_sgd", 2, 128 * 77, 128, 0.6, "sgd", "f32", "f32", LOSSLESS | SKIP),
+    ("w64_fp32", 64, 1024 * 20, 1024, 0.05, "sgd", "f32", "f32", 0),
+    ("packet_not_multiple_of_chunk", 5, 1000 * 13 + 24, 1000, 0.15, "adam", "bf16", "bf16", 0),
+]
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+@pytest.mark.parametrize("fused", [True, False])
+def test_edge_cases(case, fused):
+    name, W, n, P, p, opt, gd, rd, flags = case
+    w = workload.Workload(name, W, n, P, p, opt, 1e-2 if opt == "sgd" else 3e-4, gd, rd, 5, seed=42)
+    gpu, orc = run_parity(w, 5, fused=fused, flags=flags)
+    if name.startswith("heavy_loss"):
+        assert int((gpu.count == 0).sum()) > 0          # the nothing-received fallback was exercised
+
+
+def test_different_p_grad_and_p_param():
+    w = workload.Workload("two_rates", 6, 512 * 40, 512, 0.0, "adam", 3e-4, "bf16", "bf16", 4, seed=3)
+    run_parity(w, 4, p_grad=0.25, p_param=0.05)
+    run_parity(w, 4, p_grad=0.0, p_param=0.5, fused=False)
+
+
+def test_fused_equals_unfused_bitwise_and_without_optional_outputs():
+    w = workload.scaled(CFG["cfg2_w8_layer_adam"], 2048 * 50 + 8 * 11)
+    a, b, c = GpuRun(w), GpuRun(w), GpuRun(w)
+    for t in range(1, 6):
+        gd = [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)]
+        a.step_fused(t, gd)
+        b.step_unfused(t, gd)
+        c.step_fused(t, gd, outputs=False)
+        torch.cuda.synchronize()
+        for x, y in ((a, b), (a, c)):
+            assert torch.equal(x.master, y.master) and torch.equal(x.m, y.m) and torch.equal(x.v, y.v)
+            for i in range(w.W):
+                assert torch.equal(x.replicas[i], y.replicas[i])
+            assert torch.equal(x.norms, y.norms)
+        assert torch.equal(a.ghat, b.ghat) and torch.equal(a.count, b.count)
+        assert torch.equal(a.recv, b.recv) and torch.equal(a.stale, b.stale)
+        assert torch.equal(a.sumsq, b.sumsq)
+
+
+def test_checkpoint_resume_is_bit_identical():
+    w = workload.scaled(CFG["cfg2_w8_layer_adam"], 2048 * 20)
+    a = GpuRun(w)
+    for t in range(1, 11):
+        a.step_fused(t, [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)])
+    b = GpuRun(w)
+    for t in range(1, 6):
+        b.step_fused(t, [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)])
+    saved = [b.master.cpu(), b.m.cpu(), b.v.cpu()] + [r.cpu() for r in b.replicas]
+    b.close()
+    c = GpuRun(w)                                       # fresh context: masks are a function of (seed, step, ...)
+    c.master.copy_(saved[0]); c.m.copy_(saved[1]); c.v.copy_(saved[2])
+    for i in range(w.W):
+        c.replicas[i].copy_(saved[3 + i])
+    for t in range(6, 11):
+        c.step_fused(t, [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)])
+    torch.cuda.synchronize()
+    assert torch.equal(a.master, c.master) and torch.equal(a.v, c.v)
+    for i in range(w.W):
+        assert torch.equal(a.replicas[i], c.replicas[i])
+    assert torch.equal(a.norms, c.norms)
+
+
+def test_learning_rate_schedule():
+    w = workload.Workload("lr_sched", 4, 256 * 30, 256, 0.1, "sgd", 1e-2, "f32", "f32", 4, seed=8)
+    gpu, orc = GpuRun(w), make_oracle(w)
+    for t, lr in enumerate([1e-2, 5e-3, 2.5e-3, 0.0], start=1):
+        L.lossy_set_lr(gpu.ctx, lr)
+        orc.set_lr(lr)
+        gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]
+        gpu.step_fused(t, [g.cuda() for g in gs])
+        ref = orc.step(t, [to_np(g) for g in gs])
+        compare_outputs(gpu.outputs(), ref, f"lr step {t}")
+        compare_state(gpu, orc, f"lr step {t}")
+
+
+def test_empty_bucket_is_a_noop_and_bad_arguments_are_rejected():
+    dev = "cuda"
+    ctx = L.lossy_init(W=2, n=0, packet_elems=64, p_grad=0.1, p_param=0.1, seed=0, grad_dtype=torch.float32,
+                       replica_dtype=torch.float32, optimizer="sgd", lr=0.1)
+    z = [torch.zeros(8, device=dev) for _ in range(2)]
+    norms = torch.ones(2, device=dev)
+    L.lossy_fused_step(ctx, 1, z, z[0], None, None, z, norms=norms)
+    torch.cuda.synchronize()
+    assert float(norms.abs().sum()) == 0.0
+    assert L.lossy_kernel_launches(ctx) == 0
+    L.lossy_destroy(ctx)
+    for bad in (dict(W=0), dict(W=65), dict(packet_elems=0), dict(packet_elems=12), dict(p_grad=1.0),
+                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=8), dict(optimizer=5)):
+        kw = dict(W=2, n=64, packet_elems=64, p_grad=0.1, p_param=0.1, seed=0, grad_dtype=torch.float32,
+                  replica_dtype=torch.float32, optimizer="sgd", lr=0.1)
+        kw.update(bad)
+        with pytest.raises(L.LossyError) as ei:
+            L.lossy_init(**kw)
+        assert ei.value.code == L.LOSSY_EINVAL
+    ctx = L.lossy_init(W=2, n=64, packet_elems=64, p_grad=0.1, p_param=0.1, seed=0, grad_dtype=torch.float32,
+                       replica_dtype=torch.float32, optimizer="adam", lr=0.1)
+    g = [torch.zeros(64, device=dev) for _ in range(2)]
+    r = [torch.zeros(64, device=dev) for _ in range(2)]
+    th = torch.zeros(64, device=dev)
+    with pytest.raises(L.LossyError):                   # Adam without moments
+        L.lossy_fused_step(ctx, 1, g, th, None, None, r)
+    with pytest.raises(L.LossyError):                   # step 0
+        L.lossy_fused_step(ctx, 0, g, th, th.clone(), th.clone(), r)
+    mis = torch.zeros(80, device=dev)[1:65]             # 4-byte offset: not 16-byte aligned
+    with pytest.raises(L.LossyError):
+        L.lossy_fused_step(ctx, 1, [mis, g[1]], th, th.clone(), th.clone(), r)
+    assert L.lossy_kernel_launches(ctx) == 0            # nothing was launched for rejected calls
+    L.lossy_destroy(ctx)

@@ -1,0 +1,61 @@
+"""The C-ABI shared library builds, loads and exports every symbol include/lossy.h declares.
+No compute call is made here (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2507_07114_b200 as L
+from paper_2507_07114_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "lossy.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lossy_[a-z0-9_]+|drift_norms)\s*\(", text)))
+
+
+def test_header_symbols_are_exported_and_bound():
+    B.build()
+    lib = ctypes.CDLL(B.LIB_PATH)
+    names = _declared()
+    assert "lossy_init" in names and "drift_norms" in names and "lossy_fused_step" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in lossy.h but not exported"
+        assert n in L.EXPORTS, f"{n} has no Python binding of the same name"
+        assert callable(getattr(L, n))
+    assert sorted(L.EXPORTS) == names
+
+
+def test_config_struct_layout_matches_the_header():
+    # uint32 W, P; uint64 n, base; double x2; uint64 seed; uint32 x4; float x4
+    assert ctypes.sizeof(L.lossy_config) == 4 + 4 + 8 + 8 + 8 + 8 + 8 + 16 + 16
+    assert L.lossy_config.n.offset == 8 and L.lossy_config.seed.offset == 40 and L.lossy_config.lr.offset == 64
+
+
+def test_host_only_entry_points_work_without_a_gpu():
+    # the delivery-indicator hash is a pure host function of its arguments
+    a = L.lossy_hash_u32(1, 2, 3, 4, 5)
+    assert a == L.lossy_hash_u32(1, 2, 3, 4, 5) and a != L.lossy_hash_u32(1, 2, 4, 3, 5)
+    assert L.lossy_mask(None, 1, 0, 0, 0) == -1
+    assert L.lossy_num_packets(None) == 0
+
+
+def test_missing_library_fails_loudly():
+    with pytest.raises(FileNotFoundError):
+        L.load_library(os.path.join(ROOT, "no_such_dir", "liblossy_b200.so"))
+
+
+def test_product_path_never_touches_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2507_07114_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src.lower(), f"{f} mentions the oracle"
+    for f in ("lossy_oracle.c", "oracle.py"):
+        src = open(os.path.join(ROOT, "oracle", f)).read()
+        assert "paper_2507_07114_b200" not in src and "lossy.h" not in src

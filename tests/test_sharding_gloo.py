@@ -1,0 +1,79 @@
+"""The N>1 path on CPU: ranks take contiguous bucket ranges, run independently (no data-path
+collective) and only the per-replica squared drift sums are all-reduced. world_size 2, gloo."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import workload
+from paper_2507_07114_b200.sharding import shard_range
+from parity_util import make_oracle, to_np
+
+
+def test_shard_range_partitions_exactly():
+    for units in (0, 1, 7, 8, 34):
+        for world in (1, 2, 3, 8):
+            got = [shard_range(units, r, world) for r in range(world)]
+            assert got[0][0] == 0 and got[-1][1] == units
+            assert all(a[1] == b[0] for a, b in zip(got[:-1], got[1:]))
+            sizes = [b - a for a, b in got]
+            assert max(sizes) - min(sizes) <= 1
+
+
+BUCKETS = [512 * 9, 512 * 7 + 40, 512 * 12, 512 * 5, 512 * 3 + 8]
+
+
+def _bucket_workloads():
+    base = workload.baseline_workloads()["cfg4_w8_full_model"]
+    out, pb = [], 0
+    for b, n in enumerate(BUCKETS):
+        w = workload.scaled(base, n, packet_elems=512, packet_base=pb, name=f"bucket{b}")
+        out.append(w)
+        pb += w.K
+    return out
+
+
+def _run_buckets(ws, steps):
+    tot = np.zeros(8)
+    for w in ws:
+        o = make_oracle(w)
+        for t in range(1, steps + 1):
+            r = o.step(t, [to_np(workload.grad_slab(w, t, i, 0, w.n)) for i in range(w.W)])
+        tot += r["sumsq"]
+    return tot
+
+
+def _worker(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ws = _bucket_workloads()
+    lo, hi = shard_range(len(ws), rank, world)
+    mine = torch.from_numpy(_run_buckets(ws[lo:hi], 3))
+    dist.all_reduce(mine, op=dist.ReduceOp.SUM)          # the only exchange: W doubles
+    t = torch.tensor([1.0 + rank])
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)              # bench timing rule: max over ranks
+    if rank == 0:
+        q.put((mine.numpy(), float(t)))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_reproduce_the_single_process_drift():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got, tmax = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    want = _run_buckets(_bucket_workloads(), 3)
+    assert np.allclose(got, want, rtol=1e-12)
+    assert tmax == 2.0
