@@ -154,6 +154,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=WORKLOAD)
     ap.add_argument("--elements", type=int, default=0, help="override the bucket size (profiling of a small case)")
+    ap.add_argument("--p", type=float, default=None, help="override the drop probability")
+    ap.add_argument("--workers", type=int, default=0, help="override W")
+    ap.add_argument("--packet-elems", type=int, default=0, help="override the packet size")
     ap.add_argument("--e2e-steps", type=int, default=-1, help="steps of the host-buffer leg (default: min(steps, 10))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-packets", type=int, default=8192)
@@ -171,6 +174,12 @@ def main():
     w = workload.baseline_workloads()[args.workload]
     if args.elements:
         w = workload.scaled(w, args.elements)
+    if args.p is not None:
+        w = workload.scaled(w, w.n, p=args.p)
+    if args.workers:
+        w = workload.scaled(w, w.n, W=args.workers)
+    if args.packet_elems:
+        w = workload.scaled(w, w.n, packet_elems=args.packet_elems)
     warmup = max(3, args.warmup)
 
     if args.impl == "reference":
@@ -312,7 +321,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
                          "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured"
-                         else peak_src, "kernel": "lossy_kernel<AGG|STEP|BCAST|DRIFT> + 64-thread finalize",
+                         else peak_src, "kernel": "lossy_fused_tma_kernel (+ W-warp drift finalize)",
                          "avg_launch_ms": avg_launch_ms, "min_launch_ms": min(per_launch_ms)},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
         }

@@ -42,7 +42,7 @@ extern "C" {
 
 typedef struct lossy_ctx lossy_ctx; /* opaque; host object + small device scratch */
 
-enum { LOSSY_OK = 0, LOSSY_EINVAL = 1, LOSSY_ENOMEM = 2, LOSSY_ECUDA = 3 };
+enum { LOSSY_OK = 0, LOSSY_EINVAL = 1, LOSSY_ENOMEM = 2, LOSSY_ECUDA = 3, LOSSY_EDEVICE = 4 };
 enum { LOSSY_F32 = 0, LOSSY_BF16 = 1 };  /* element types of gradients / replicas */
 enum { LOSSY_SGD = 0, LOSSY_ADAM = 1 };
 enum {
@@ -52,7 +52,10 @@ enum {
   LOSSY_SELF_LOSSLESS = 1u,
   /* A packet that received nothing leaves theta, m, v untouched. Default: the
    * estimate is exactly 0 and is fed to the unmodified optimizer. */
-  LOSSY_ZERO_SKIP = 2u
+  LOSSY_ZERO_SKIP = 2u,
+  /* lossy_fused_step always uses the register-path kernel. Default: complete packets of at
+   * least 1024 elements go through the bulk-copy (TMA) pipeline. Both give the same state. */
+  LOSSY_REGISTER_PATH = 4u
 };
 
 #define LOSSY_MAX_WORKERS 64u
@@ -68,7 +71,7 @@ typedef struct {
   uint32_t grad_dtype;   /* LOSSY_F32 or LOSSY_BF16                                     */
   uint32_t replica_dtype;/* LOSSY_F32 or LOSSY_BF16 (bf16 = round-to-nearest-even cast) */
   uint32_t optimizer;    /* LOSSY_SGD or LOSSY_ADAM                                     */
-  uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP                  */
+  uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH */
   float lr, beta1, beta2, eps; /* eta_t and Adam's constants (beta/eps unused for SGD)  */
 } lossy_config;
 
@@ -151,8 +154,10 @@ int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas
 /*
  * lossy_fused_step — steps (2), (3), (4) and the drift norms in ONE pass over
  * the bucket; ghat is not materialised unless asked for. The state it leaves
- * (master, m, v, replicas) and every optional output are bit-identical to the
- * sequence lossy_aggregate -> lossy_step -> lossy_broadcast -> drift_norms.
+ * (master, m, v, replicas), ghat, the counts and the bit sets are bit-identical
+ * to the sequence lossy_aggregate -> lossy_step -> lossy_broadcast ->
+ * drift_norms; the norms agree up to the rounding of a different (but fixed)
+ * summation order.
  * Optional outputs (NULL to skip): ghat [n], count [K], recv_bits [K],
  * stale_bits [K], norms [W], sumsq [W] (added to, as in drift_norms).
  */
@@ -166,7 +171,7 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads,
  * HOST memory (pinned memory for full copy speed): copies worker i's gradient
  * from host_grads[i] into dev_grads[i] on `stream`, runs lossy_fused_step, and
  * copies the W norms to `host_norms`. It returns after the stream has been
- * synchronised, so `host_norms` is valid on return.
+ * synchronised (through lossy_device_status), so `host_norms` is valid on return.
  *   host_grads  host array of W HOST pointers, each [n] of cfg.grad_dtype
  *   dev_grads   host array of W DEVICE staging pointers, each [n], caller-owned
  *   dev_norms   [W] fp32 device; host_norms [W] fp32 host
@@ -175,6 +180,15 @@ int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host
                           void* const* dev_grads, float* master, float* m, float* v,
                           void* const* replicas, float* dev_norms, float* host_norms,
                           void* stream);
+
+/*
+ * lossy_device_status — synchronise `stream` and report whether any kernel of
+ * this context gave up a bounded wait (the bulk-copy pipeline bounds every wait
+ * on its barriers instead of spinning forever). LOSSY_OK, or LOSSY_EDEVICE if
+ * the results of an earlier call on this context must be discarded. The paper
+ * has no counterpart; this is the library's failure report.
+ */
+int lossy_device_status(lossy_ctx* ctx, void* stream);
 
 /*
  * lossy_mask — host evaluation of one delivery indicator of Section 3:

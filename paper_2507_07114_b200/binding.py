@@ -14,15 +14,15 @@ import torch
 
 from . import build as _build
 
-LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA = 0, 1, 2, 3
+LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE = 0, 1, 2, 3, 4
 LOSSY_F32, LOSSY_BF16 = 0, 1
 LOSSY_SGD, LOSSY_ADAM = 0, 1
-LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP = 1, 2
+LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_aggregate", "lossy_step", "lossy_broadcast",
     "drift_norms", "lossy_fused_step", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
-    "lossy_mask_grid", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
+    "lossy_mask_grid", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
 
 
@@ -80,6 +80,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_hash_u32.argtypes = [u64, u64, u32, u32, u64]
     lib.lossy_mask_grid.restype = C.c_int
     lib.lossy_mask_grid.argtypes = [vp, u64, vp, vp, vp, u64, C.c_int, vp, vp]
+    lib.lossy_device_status.restype = C.c_int
+    lib.lossy_device_status.argtypes = [vp, vp]
     lib.lossy_last_error.restype = C.c_char_p
     lib.lossy_last_error.argtypes = [vp]
     lib.lossy_num_packets.restype = u64
@@ -182,6 +184,11 @@ def lossy_hash_u32(seed, step, src, dst, packet) -> int:
 def lossy_mask_grid(ctx, step, src, dst, packet, out, is_param=False):
     _check(ctx, load_library().lossy_mask_grid(ctx, step, _p(src), _p(dst), _p(packet), src.numel(), int(is_param),
                                                _p(out), _stream()))
+
+
+def lossy_device_status(ctx):
+    """Synchronise the current stream; raises LossyError(LOSSY_EDEVICE) if a kernel gave up a bounded wait."""
+    _check(ctx, load_library().lossy_device_status(ctx, _stream()))
 
 
 def lossy_last_error(ctx) -> str:

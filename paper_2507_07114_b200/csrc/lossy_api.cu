@@ -8,7 +8,7 @@
 
 #include <new>
 
-#include "lossy_kernels.cuh"
+#include "lossy_tma.cuh"
 
 using namespace lossy;
 
@@ -22,7 +22,9 @@ struct lossy_ctx {
   int device;
   int num_sms;
   uint32_t max_blocks;   // capacity of `partials`
-  double* partials;      // device, [max_blocks][kMaxW]
+  double* partials;      // device, [max_blocks][kMaxW], followed by the status word
+  uint32_t* status;      // device status word: 0 = fine, 1 = a bounded wait in a kernel gave up
+  int smem_optin;        // largest dynamic shared memory a block may opt in to
   uint64_t launches;
   char err[256];
 };
@@ -75,6 +77,66 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   P.partials = ctx->partials;
 }
 
+// ---- bulk-copy pipeline (fused step only) --------------------------------------------------
+constexpr uint32_t kTmaSmemBudget = 112 * 1024;   // two CTAs per SM
+constexpr uint32_t kTmaSmemFixed = 128 + kMaxStages * sizeof(StageHdr);
+
+bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
+  const lossy_config& c = ctx->cfg;
+  if (c.flags & LOSSY_REGISTER_PATH) return false;
+  if (c.packet_elems < (uint32_t)kTile) return false;        // small packets: the register kernel
+  const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
+  if (kfull == 0) return false;
+  const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
+  G.grad_slots = c.W < (uint32_t)kGroup ? c.W : (uint32_t)kGroup;
+  G.groups = (c.W + kGroup - 1) / kGroup;
+  uint32_t sb = G.grad_slots * kTile * gb + 3 * kTile * 4 + kTile * rb;
+  G.stage_bytes = (sb + 127u) & ~127u;
+  uint32_t budget = kTmaSmemBudget;
+  if ((uint32_t)ctx->smem_optin < budget) budget = (uint32_t)ctx->smem_optin;
+  if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
+  G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
+  if (G.stages > (uint32_t)kMaxStages) G.stages = kMaxStages;
+  G.tiles_per_packet = (c.packet_elems + kTile - 1) / kTile;
+  const uint64_t tiles = kfull * G.tiles_per_packet;
+  if (tiles >= (1ull << 31)) return false;
+  G.num_tiles = (uint32_t)tiles;
+  G.status = ctx->status;
+  return true;
+}
+
+template <class GT, class RT, int OPT, bool DRIFTK>
+int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
+  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK>;
+  const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kTmaThreads, smem);
+  if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
+  if (per_sm < 1) per_sm = 1;
+  if (per_sm > 2) per_sm = 2;
+  uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
+  if (blocks > G.num_tiles) blocks = G.num_tiles;
+  kern<<<blocks, kTmaThreads, smem, s>>>(P, G);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "bulk-copy kernel launch", e);
+  ctx->launches++;
+  *blocks_out = blocks;
+  return LOSSY_OK;
+}
+
+template <bool DRIFTK>
+int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
+  const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
+  const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
+  const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
+  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK>(ctx, P, G, s, blocks);
+  return adam ? launch_tma<F32, F32, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK>(ctx, P, G, s, blocks);
+}
+
 template <int PH, class GT, class RT, int OPT>
 int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out) {
   auto kern = lossy_kernel<PH, GT, RT, OPT>;
@@ -84,9 +146,9 @@ int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out
   if (per_sm < 1) per_sm = 1;
   if (per_sm > kBlocksPerSmCap) per_sm = kBlocksPerSmCap;
   uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
-  const uint32_t need = (P.num_chunks + kWarps - 1) / kWarps;
+  const uint32_t need = (P.num_chunks - P.chunk_begin + kWarps - 1) / kWarps;
   if (blocks > need) blocks = need;
-  if (blocks > ctx->max_blocks) blocks = ctx->max_blocks;
+  if (blocks > ctx->max_blocks - P.partials_row0) blocks = ctx->max_blocks - P.partials_row0;
   if (blocks == 0) blocks = 1;
   kern<<<blocks, kThreads, 0, s>>>(P);
   e = cudaGetLastError();
@@ -97,7 +159,7 @@ int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out
 }
 
 int finalize_drift(lossy_ctx* ctx, uint32_t blocks, float* norms, double* sumsq, cudaStream_t s) {
-  drift_finalize_kernel<<<1, kMaxW, 0, s>>>(ctx->partials, blocks, ctx->cfg.W, norms, sumsq);
+  drift_finalize_kernel<<<ctx->cfg.W, 32, 0, s>>>(ctx->partials, blocks, ctx->cfg.W, norms, sumsq);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda(ctx, "drift finalize launch", e);
   ctx->launches++;
@@ -135,7 +197,7 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   if (cfg->packet_elems == 0 || cfg->packet_elems % 8 != 0) return LOSSY_EINVAL;
   if (!(cfg->p_grad >= 0.0 && cfg->p_grad < 1.0) || !(cfg->p_param >= 0.0 && cfg->p_param < 1.0)) return LOSSY_EINVAL;
   if (cfg->grad_dtype > LOSSY_BF16 || cfg->replica_dtype > LOSSY_BF16 || cfg->optimizer > LOSSY_ADAM) return LOSSY_EINVAL;
-  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP)) return LOSSY_EINVAL;
+  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH)) return LOSSY_EINVAL;
   const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
   const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;
   if (K * cpp >= (1ull << 31)) return LOSSY_EINVAL;  // stream larger models bucket by bucket
@@ -155,8 +217,14 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
   if (e != cudaSuccess) { delete ctx; return LOSSY_ECUDA; }
   ctx->max_blocks = (uint32_t)(ctx->num_sms * kBlocksPerSmCap);
-  e = cudaMalloc(&ctx->partials, (size_t)ctx->max_blocks * kMaxW * sizeof(double));
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device);
+  if (e != cudaSuccess) { delete ctx; return LOSSY_ECUDA; }
+  const size_t pbytes = (size_t)ctx->max_blocks * kMaxW * sizeof(double);
+  e = cudaMalloc(&ctx->partials, pbytes + 256);
   if (e != cudaSuccess) { delete ctx; return e == cudaErrorMemoryAllocation ? LOSSY_ENOMEM : LOSSY_ECUDA; }
+  ctx->status = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(ctx->partials) + pbytes);
+  e = cudaMemset(ctx->status, 0, 256);
+  if (e != cudaSuccess) { cudaFree(ctx->partials); delete ctx; return LOSSY_ECUDA; }
   *out = ctx;
   return LOSSY_OK;
 }
@@ -274,12 +342,33 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, fl
   P.recv_bits = recv_bits;
   P.stale_bits = stale_bits;
   cudaStream_t s = (cudaStream_t)stream;
-  if (norms || sumsq) {
+  const bool drift = norms || sumsq;
+  uint32_t rows = 0;
+  TmaGeom G;
+  if (tma_geometry(ctx, G)) {
+    // complete packets go through the bulk-copy pipeline, a short last packet through the register kernel
     uint32_t blocks = 0;
-    if (int rc = dispatch<AGG | STEP | BCAST | DRIFT>(ctx, P, s, &blocks)) return rc;
-    return finalize_drift(ctx, blocks, norms, sumsq, s);
+    if (int rc = drift ? dispatch_tma<true>(ctx, P, G, s, &blocks) : dispatch_tma<false>(ctx, P, G, s, &blocks)) return rc;
+    rows = blocks;
+    P.chunk_begin = (uint32_t)((ctx->cfg.n / ctx->cfg.packet_elems) * ctx->chunks_per_packet);
+    P.partials_row0 = rows;
   }
-  return dispatch<AGG | STEP | BCAST>(ctx, P, s, nullptr);
+  if (P.chunk_begin < P.num_chunks) {
+    uint32_t blocks = 0;
+    if (int rc = drift ? dispatch<AGG | STEP | BCAST | DRIFT>(ctx, P, s, &blocks) : dispatch<AGG | STEP | BCAST>(ctx, P, s, &blocks)) return rc;
+    rows += blocks;
+  }
+  return drift ? finalize_drift(ctx, rows, norms, sumsq, s) : LOSSY_OK;
+}
+
+int lossy_device_status(lossy_ctx* ctx, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  uint32_t word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, ctx->status, sizeof word, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(ctx, "status read", e);
+  if (word != 0) return fail(ctx, LOSSY_EDEVICE, "a bounded wait inside a kernel gave up; results of that call are invalid");
+  return LOSSY_OK;
 }
 
 int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host_grads, void* const* dev_grads,
@@ -301,9 +390,7 @@ int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host
     return rc;
   cudaError_t e = cudaMemcpyAsync(host_norms, dev_norms, ctx->cfg.W * sizeof(float), cudaMemcpyDeviceToHost, s);
   if (e != cudaSuccess) return fail_cuda(ctx, "norm download", e);
-  e = cudaStreamSynchronize(s);
-  if (e != cudaSuccess) return fail_cuda(ctx, "stream synchronize", e);
-  return LOSSY_OK;
+  return lossy_device_status(ctx, stream);   // synchronises the stream
 }
 
 uint32_t lossy_hash_u32(uint64_t seed, uint64_t step, uint32_t src, uint32_t dst, uint64_t packet) {

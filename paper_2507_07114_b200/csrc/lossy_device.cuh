@@ -14,7 +14,13 @@
 namespace lossy {
 
 constexpr int kMaxW = 64;
-constexpr int kThreads = 256;
+#ifndef LOSSY_THREADS
+#define LOSSY_THREADS 256
+#endif
+#ifndef LOSSY_MIN_BLOCKS
+#define LOSSY_MIN_BLOCKS 1
+#endif
+constexpr int kThreads = LOSSY_THREADS;
 constexpr int kWarps = kThreads / 32;
 constexpr int kChunk = 256;  // elements per warp-chunk
 
@@ -36,6 +42,8 @@ struct Params {
   uint64_t packet_base;
   uint64_t step_key;      // hash key of (seed, step), derived on the host
   uint32_t num_chunks;    // K * chunks_per_packet
+  uint32_t chunk_begin;   // first chunk this launch covers (a bulk-copy launch may own the chunks before it)
+  uint32_t partials_row0; // first row of `partials` this launch writes
   uint32_t chunks_per_packet;
   uint32_t pps;           // packets per shard
   uint32_t P;

@@ -27,8 +27,36 @@ __device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8],
   }
 }
 
+// Delivery indicators of packet k (owner j), evaluated one worker per lane and gathered by ballot:
+// recv bit i = gradient piece of worker i reached the owner; stale bit i = replica i missed the broadcast.
+template <int PH>
+__device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32_t j, int lane, uint64_t& recv,
+                                             uint64_t& stale) {
+  const uint32_t W = P.W;
+  const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k);
+  const uint32_t i0 = lane, i1 = lane + 32;
+  if constexpr (PH & AGG) {
+    bool s0 = i0 < W && (pair_hash(pkey, i0, j) >= P.Tg || ((P.flags & 1u) && i0 == j));
+    uint32_t lo = __ballot_sync(0xFFFFFFFFu, s0), hi = 0;
+    if (W > 32) {
+      bool s1 = i1 < W && (pair_hash(pkey, i1, j) >= P.Tg || ((P.flags & 1u) && i1 == j));
+      hi = __ballot_sync(0xFFFFFFFFu, s1);
+    }
+    recv = ((uint64_t)hi << 32) | lo;
+  }
+  if constexpr (PH & BCAST) {
+    bool d0 = i0 < W && i0 != j && pair_hash(pkey, j, i0) < P.Tp;
+    uint32_t lo = __ballot_sync(0xFFFFFFFFu, d0), hi = 0;
+    if (W > 32) {
+      bool d1 = i1 < W && i1 != j && pair_hash(pkey, j, i1) < P.Tp;
+      hi = __ballot_sync(0xFFFFFFFFu, d1);
+    }
+    stale = ((uint64_t)hi << 32) | lo;
+  }
+}
+
 template <int PH, class GT, class RT, int OPT>
-__global__ void __launch_bounds__(kThreads) lossy_kernel(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const __grid_constant__ Params P) {
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const uint32_t W = P.W;
@@ -37,7 +65,7 @@ __global__ void __launch_bounds__(kThreads) lossy_kernel(const __grid_constant__
   double dacc0 = 0.0, dacc1 = 0.0;
 
   const uint32_t warps_in_grid = gridDim.x * kWarps;
-  for (uint32_t q = blockIdx.x * kWarps + warp; q < P.num_chunks; q += warps_in_grid) {
+  for (uint32_t q = P.chunk_begin + blockIdx.x * kWarps + warp; q < P.num_chunks; q += warps_in_grid) {
     const uint32_t k = q / P.chunks_per_packet;
     const uint32_t c = q - k * P.chunks_per_packet;
     const uint32_t j = k / P.pps;  // owner W_j of packet k
@@ -47,28 +75,40 @@ __global__ void __launch_bounds__(kThreads) lossy_kernel(const __grid_constant__
     if (in_pkt < P.P && e < P.n) nvalid = (P.n - e >= 8) ? 8 : (int)(P.n - e);
 
     // ---- delivery indicators of this packet (warp-uniform) -------------------
-    const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k);
     uint64_t recv = 0, stale = 0;
-    if constexpr (PH & AGG) {
-      const uint32_t i0 = lane, i1 = lane + 32;
-      bool s0 = i0 < W && (pair_hash(pkey, i0, j) >= P.Tg || ((P.flags & 1u) && i0 == j));
-      uint32_t lo = __ballot_sync(0xFFFFFFFFu, s0), hi = 0;
-      if (W > 32) {
-        bool s1 = i1 < W && (pair_hash(pkey, i1, j) >= P.Tg || ((P.flags & 1u) && i1 == j));
-        hi = __ballot_sync(0xFFFFFFFFu, s1);
+    packet_masks<PH>(P, k, j, lane, recv, stale);
+#ifndef LOSSY_NO_PREFETCH
+    // pull the NEXT chunk of this warp toward L2 while this one is processed
+    {
+      const uint32_t qn = q + warps_in_grid;
+      if (qn < P.num_chunks) {
+        const uint32_t kn = qn / P.chunks_per_packet;
+        const uint32_t cn = qn - kn * P.chunks_per_packet;
+        const uint32_t inn = cn * kChunk + lane * 8;
+        const uint64_t en = (uint64_t)kn * P.P + inn;
+        uint64_t rn = 0, sn = 0;
+        packet_masks<PH>(P, kn, kn / P.pps, lane, rn, sn);
+        if (inn < P.P && en + 8 <= P.n) {
+          if constexpr (PH & (STEP | BCAST | DRIFT)) prefetch_l2(P.master + en);
+          if constexpr ((PH & STEP) && OPT == 1) { prefetch_l2(P.m + en); prefetch_l2(P.v + en); }
+          if constexpr (PH & AGG) {
+            while (rn) {
+              const int i = __ffsll((long long)rn) - 1;
+              rn &= rn - 1;
+              prefetch_l2(reinterpret_cast<const typename GT::raw*>(P.grads[i]) + en);
+            }
+          }
+          if constexpr ((PH & BCAST) && (PH & DRIFT)) {
+            while (sn) {
+              const int i = __ffsll((long long)sn) - 1;
+              sn &= sn - 1;
+              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + en);
+            }
+          }
+        }
       }
-      recv = ((uint64_t)hi << 32) | lo;
     }
-    if constexpr (PH & BCAST) {
-      const uint32_t i0 = lane, i1 = lane + 32;
-      bool d0 = i0 < W && i0 != j && pair_hash(pkey, j, i0) < P.Tp;
-      uint32_t lo = __ballot_sync(0xFFFFFFFFu, d0), hi = 0;
-      if (W > 32) {
-        bool d1 = i1 < W && i1 != j && pair_hash(pkey, j, i1) < P.Tp;
-        hi = __ballot_sync(0xFFFFFFFFu, d1);
-      }
-      stale = ((uint64_t)hi << 32) | lo;
-    }
+#endif
     uint32_t cnt = __popcll(recv);
     if (c == 0 && lane == 0) {
       if constexpr (PH & AGG) {
@@ -160,27 +200,44 @@ __global__ void __launch_bounds__(kThreads) lossy_kernel(const __grid_constant__
       const Vec8<RT> wire = narrow<RT>(th);
       float xw[8];
       widen<RT>(wire, xw);
-      for (uint32_t i = 0; i < W; ++i) {
-        const bool is_stale = (stale >> i) & 1ull;
-        if constexpr (PH & BCAST) {
-          if (!is_stale) {
-            store8<RT>(P.replicas[i], e, wire, nvalid);
-            continue;
-          }
-        }
-        if constexpr (PH & DRIFT) {
-          const Vec8<RT> old = load8_any<RT>(P.replicas[i], e, nvalid);
-          float fo[8];
-          widen<RT>(old, fo);
-          float s = 0.0f;
+      if constexpr (PH & BCAST) {
+        for (uint32_t i = 0; i < W; ++i)
+          if (!((stale >> i) & 1ull)) store8<RT>(P.replicas[i], e, wire, nvalid);
+      }
+      if constexpr (PH & DRIFT) {
+        // copies that differ from the wire value: the stale ones after a broadcast, or (standalone) all
+        uint64_t todo = (PH & BCAST) ? stale : (W == 64 ? ~0ull : ((1ull << W) - 1ull));
+        while (todo) {
+          // up to four copies are fetched before the first is used
+          int ids[4];
+          Vec8<RT> old[4];
+          int nb = 0;
 #pragma unroll
-          for (int x = 0; x < 8; ++x) {
-            const float d = x < nvalid ? __fsub_rn(fo[x], xw[x]) : 0.0f;
-            s = __fadd_rn(s, __fmul_rn(d, d));
+          for (int b = 0; b < 4; ++b) {
+            ids[b] = -1;
+            if (todo) {
+              ids[b] = __ffsll((long long)todo) - 1;
+              todo &= todo - 1;
+              nb = b + 1;
+              old[b] = load8_any<RT>(P.replicas[ids[b]], e, nvalid);
+            }
           }
-          const float tot = warp_sum(s);
-          if ((i & 31u) == (uint32_t)lane) {
-            if (i < 32) dacc0 += (double)tot; else dacc1 += (double)tot;
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            if (b < nb) {
+              float fo[8];
+              widen<RT>(old[b], fo);
+              float s = 0.0f;
+#pragma unroll
+              for (int x = 0; x < 8; ++x) {
+                const float d = x < nvalid ? __fsub_rn(fo[x], xw[x]) : 0.0f;
+                s = __fadd_rn(s, __fmul_rn(d, d));
+              }
+              const float tot = warp_sum(s);
+              if ((ids[b] & 31) == lane) {
+                if (ids[b] < 32) dacc0 += (double)tot; else dacc1 += (double)tot;
+              }
+            }
           }
         }
       }
@@ -197,20 +254,25 @@ __global__ void __launch_bounds__(kThreads) lossy_kernel(const __grid_constant__
       double t = 0.0;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) t += sh[w][threadIdx.x];
-      P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
+      P.partials[(size_t)(P.partials_row0 + blockIdx.x) * kMaxW + threadIdx.x] = t;
     }
   }
 }
 
-// Sum the per-block partials in block order; add to sumsq, write the norms.
+// Sum the per-block partials of replica blockIdx.x in a fixed order (lane l takes rows l, l+32, ...,
+// then a shuffle tree); add to sumsq, write the norm. One warp per replica.
 __global__ void drift_finalize_kernel(const double* __restrict__ partials, uint32_t nblocks, uint32_t W,
                                       float* norms, double* sumsq) {
-  const uint32_t i = threadIdx.x;
+  const uint32_t i = blockIdx.x;
   if (i >= W) return;
   double t = 0.0;
-  for (uint32_t b = 0; b < nblocks; ++b) t += partials[(size_t)b * kMaxW + i];
-  if (sumsq) sumsq[i] += t;
-  if (norms) norms[i] = (float)sqrt(t);
+  for (uint32_t b = threadIdx.x; b < nblocks; b += 32) t += partials[(size_t)b * kMaxW + i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+  if (threadIdx.x == 0) {
+    if (sumsq) sumsq[i] += t;
+    if (norms) norms[i] = (float)sqrt(t);
+  }
 }
 
 // Delivery indicators on a dense grid of tuples (host/device agreement check).

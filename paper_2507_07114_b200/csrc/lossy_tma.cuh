@@ -1,0 +1,410 @@
+// Fused lossy step as a bulk-copy (TMA) pipeline for sm_100a.
+//
+// One CTA = kConsumerWarps compute warps + 1 producer warp + 1 store warp, two CTAs per SM.
+// The bucket's full packets are cut into tiles of at most kTile contiguous elements inside one
+// packet, so one set of delivery masks covers a tile. Per tile and per group of up to 8 workers
+// the producer arms an mbarrier and issues 1-D bulk copies global -> shared memory for the
+// DELIVERED workers' pieces only (dropped packets are never read) and, with the last group, for
+// theta / m / v. Compute warps sum the pieces in ascending worker order from shared memory,
+// divide by the received count, run the optimizer in place in shared memory and write the wire
+// value (fp32 or RNE bf16) once; the store warp then fans that single shared-memory tile out with
+// one bulk copy per replica that receives the broadcast, plus theta / m / v. Replicas that miss
+// the broadcast are not written; their old packet is read (L2-prefetched by the producer) only to
+// accumulate the drift term. No cluster launch and no multicast: the path has no cross-CTA reuse.
+//
+// Every wait on an mbarrier is bounded: after kMaxPolls unsuccessful polls the CTA raises a
+// shared abort flag, records a code in the context's device status word and every role leaves
+// its loop; the producer then gives its own copies in flight a bounded time to land.
+#pragma once
+#include "lossy_kernels.cuh"
+
+namespace lossy {
+
+constexpr int kConsumerWarps = 8;
+constexpr int kEpl = 4;                                   // elements per compute lane
+constexpr int kTile = kConsumerWarps * 32 * kEpl;         // 1024 elements
+constexpr int kTmaThreads = (kConsumerWarps + 2) * 32;    // + producer warp + store warp
+constexpr int kGroup = 8;                                 // workers per pipeline stage
+constexpr int kMaxStages = 4;
+constexpr uint32_t kMaxPolls = 1u << 22;
+
+struct TmaGeom {
+  uint32_t num_tiles;         // full packets * tiles_per_packet
+  uint32_t tiles_per_packet;
+  uint32_t stages;
+  uint32_t stage_bytes;       // per stage, 128-byte multiple
+  uint32_t groups;            // ceil(W / kGroup)
+  uint32_t grad_slots;        // min(W, kGroup)
+  uint32_t* status;           // device status word (0 = fine)
+};
+
+struct __align__(16) StageHdr {
+  uint64_t recv, stale, e0;
+  uint32_t k, len, cnt, last;
+  uint32_t pad[6];
+};
+static_assert(sizeof(StageHdr) == 64, "header is one 64-byte slot");
+
+// ---- PTX wrappers ---------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Bounded wait; false = gave up (or another role already aborted).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u && *abort_flag) return false;
+  }
+  *abort_flag = 1u;
+  return false;
+}
+
+template <class T, int N> struct LaneVec;   // N elements of type T as one shared-memory access
+template <> struct LaneVec<F32, 4> { using type = uint4; };
+template <> struct LaneVec<BF16, 4> { using type = uint2; };
+
+template <class T>
+__device__ __forceinline__ void lds4(const unsigned char* base, uint32_t idx, float (&f)[4]) {
+  if constexpr (T::kVecs == 2) {
+    const uint4 r = *reinterpret_cast<const uint4*>(base + (size_t)idx * 4);
+    f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y); f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+  } else {
+    const uint2 r = *reinterpret_cast<const uint2*>(base + (size_t)idx * 2);
+    f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xFFFF0000u);
+    f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xFFFF0000u);
+  }
+}
+__device__ __forceinline__ void sts4_f32(unsigned char* base, uint32_t idx, const float (&f)[4]) {
+  *reinterpret_cast<uint4*>(base + (size_t)idx * 4) =
+      make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+}
+__device__ __forceinline__ uint2 pack_bf16x4(const float (&f)[4]) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]);
+  __nv_bfloat162 b = __floats2bfloat162_rn(f[2], f[3]);
+  return make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+}
+
+template <class GT, class RT, int OPT, bool DRIFTK>
+__global__ void __launch_bounds__(kTmaThreads, 2) lossy_fused_tma_kernel(const __grid_constant__ Params P,
+                                                                         const __grid_constant__ TmaGeom G) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
+  // layout: [full, done, empty barriers | abort flag] (128 B) | headers (kMaxStages x 64 B) | stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 96);
+  StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + 128);
+  unsigned char* stage0 = smem + 128 + kMaxStages * sizeof(StageHdr);
+  const uint32_t S = G.stages;
+  const uint32_t off_th = G.grad_slots * kTile * kGB;
+  const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4, off_wire = off_v + kTile * 4;
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const uint32_t W = P.W;
+  auto full_bar = [&](uint32_t s) { return smem_u32(&bars[s]); };
+  auto done_bar = [&](uint32_t s) { return smem_u32(&bars[kMaxStages + s]); };
+  auto empty_bar = [&](uint32_t s) { return smem_u32(&bars[2 * kMaxStages + s]); };
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    for (uint32_t s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(done_bar(s), kConsumerWarps);
+      mbar_init(empty_bar(s), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  __syncthreads();
+
+  double dacc0 = 0.0, dacc1 = 0.0;   // compute warps: lane l holds replicas l and l + 32
+
+  if (warp == kConsumerWarps) {
+    // =============================== producer warp ===============================
+    uint32_t it = 0, armed_mask = 0, armed_par = 0;
+    bool ok = true;
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      const uint32_t k = tile / G.tiles_per_packet;
+      const uint32_t c = tile - k * G.tiles_per_packet;
+      const uint32_t j = k / P.pps;
+      const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
+      const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
+      uint64_t recv = 0, stale = 0;
+      packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale);
+      const uint32_t cnt = __popcll(recv);
+      if (c == 0 && lane == 0) {
+        if (P.count) P.count[k] = (uint8_t)cnt;
+        if (P.recv_bits) P.recv_bits[k] = recv;
+        if (P.stale_bits) P.stale_bits[k] = stale;
+      }
+      if constexpr (DRIFTK) {
+        for (uint32_t i = lane; i < W; i += 32)
+          if ((stale >> i) & 1ull)
+            bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
+      }
+      for (uint32_t g = 0; g < G.groups; ++g, ++it) {
+        const uint32_t s = it % S, par = (it / S) & 1u;
+        if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
+        const bool last = g + 1 == G.groups;
+        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & 0xFFu;
+        unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+        if (lane == 0) {
+          StageHdr& h = hdrs[s];
+          h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
+          uint32_t bytes = __popc(bits) * len * kGB;
+          if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
+          mbar_arrive_expect_tx(full_bar(s), bytes);
+        }
+        __syncwarp();
+        if (lane < kGroup && ((bits >> lane) & 1u))
+          bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
+                   reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s));
+        if (last) {
+          if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s));
+          if constexpr (OPT == 1) {
+            if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s));
+            if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s));
+          }
+        }
+        armed_mask |= 1u << s;
+        armed_par = (armed_par & ~(1u << s)) | (par << s);
+      }
+    }
+    if (!ok || *abort_flag) {
+      // give this CTA's copies in flight a bounded time to land before the CTA exits
+      for (uint32_t s = 0; s < S; ++s)
+        if ((armed_mask >> s) & 1u)
+          for (uint32_t i = 0; i < (1u << 16); ++i)
+            if (mbar_try_wait(full_bar(s), (armed_par >> s) & 1u)) break;
+    }
+  } else if (warp == kConsumerWarps + 1) {
+    // ================================ store warp =================================
+    uint32_t it = 0;
+    bool ok = true;
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      for (uint32_t g = 0; g < G.groups; ++g, ++it) {
+        const uint32_t s = it % S, par = (it / S) & 1u;
+        if (!mbar_wait(done_bar(s), par, abort_flag)) { ok = false; break; }
+        if (g + 1 == G.groups) {
+          const StageHdr& h = hdrs[s];
+          const uint64_t e0 = h.e0, stale = h.stale;
+          const uint32_t len = h.len;
+          unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+          if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u);
+          if constexpr (OPT == 1) {
+            if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u);
+            if (lane == 2) bulk_s2g(P.v + e0, smem_u32(st + off_v), len * 4u);
+          }
+          for (uint32_t i = lane; i < W; i += 32)
+            if (!((stale >> i) & 1ull))
+              bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB);
+          bulk_commit();
+          bulk_wait_read0();          // shared memory of this stage may be overwritten after this
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(s));
+      }
+    }
+    bulk_wait0();
+  } else {
+    // =============================== compute warps ===============================
+    const uint32_t idx = threadIdx.x * kEpl;   // first element of this lane within the tile
+    uint32_t it = 0;
+    bool ok = true;
+    float acc[kEpl];
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      for (uint32_t g = 0; g < G.groups; ++g, ++it) {
+        const uint32_t s = it % S, par = (it / S) & 1u;
+        if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
+        const StageHdr& h = hdrs[s];
+        const uint64_t recv = h.recv;
+        const uint32_t len = h.len;
+        const bool active = idx < len;
+        unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+        if (g == 0) {
+#pragma unroll
+          for (int x = 0; x < kEpl; ++x) acc[x] = 0.0f;
+        }
+        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & 0xFFu;
+        if (active) {
+#pragma unroll
+          for (int u = 0; u < kGroup; ++u)
+            if ((bits >> u) & 1u) {
+              float f[kEpl];
+              lds4<GT>(st + (size_t)u * kTile * kGB, idx, f);
+#pragma unroll
+              for (int x = 0; x < kEpl; ++x) acc[x] = __fadd_rn(acc[x], f[x]);
+            }
+        }
+        if (g + 1 < G.groups) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(done_bar(s));
+          continue;
+        }
+        // ---- last group of the tile: estimate, update, wire value -----------------
+        const uint32_t cnt = h.cnt;
+        const uint64_t stale = h.stale, e0 = h.e0;
+        float wire[kEpl];
+        if (active) {
+          if (cnt > 0) {
+            const float fc = (float)cnt;
+#pragma unroll
+            for (int x = 0; x < kEpl; ++x) acc[x] = __fdiv_rn(acc[x], fc);
+          }
+          if (P.ghat)
+            __stcs(reinterpret_cast<uint4*>(P.ghat + e0 + idx),
+                   make_uint4(__float_as_uint(acc[0]), __float_as_uint(acc[1]), __float_as_uint(acc[2]),
+                              __float_as_uint(acc[3])));
+          float th[kEpl], m[kEpl], v[kEpl];
+          lds4<F32>(st + off_th, idx, th);
+          if (!((P.flags & 2u) && cnt == 0)) {
+            if constexpr (OPT == 1) {
+              lds4<F32>(st + off_m, idx, m);
+              lds4<F32>(st + off_v, idx, v);
+            }
+#pragma unroll
+            for (int x = 0; x < kEpl; ++x) {
+              if constexpr (OPT == 0) {
+                th[x] = __fsub_rn(th[x], __fmul_rn(P.lr, acc[x]));
+              } else {
+                const float mn = __fadd_rn(__fmul_rn(P.b1, m[x]), __fmul_rn(P.omb1, acc[x]));
+                const float vn = __fadd_rn(__fmul_rn(P.b2, v[x]), __fmul_rn(__fmul_rn(P.omb2, acc[x]), acc[x]));
+                const float mh = __fmul_rn(mn, P.ibc1);
+                const float vh = __fmul_rn(vn, P.ibc2);
+                const float den = __fadd_rn(__fsqrt_rn(vh), P.eps);
+                th[x] = __fsub_rn(th[x], __fdiv_rn(__fmul_rn(P.lr, mh), den));
+                m[x] = mn;
+                v[x] = vn;
+              }
+            }
+            sts4_f32(st + off_th, idx, th);
+            if constexpr (OPT == 1) {
+              sts4_f32(st + off_m, idx, m);
+              sts4_f32(st + off_v, idx, v);
+            }
+          }
+          if constexpr (RT::kVecs == 2) {
+            sts4_f32(st + off_wire, idx, th);
+#pragma unroll
+            for (int x = 0; x < kEpl; ++x) wire[x] = th[x];
+          } else {
+            const uint2 w2 = pack_bf16x4(th);
+            *reinterpret_cast<uint2*>(st + off_wire + (size_t)idx * 2) = w2;
+            wire[0] = __uint_as_float(w2.x << 16); wire[1] = __uint_as_float(w2.x & 0xFFFF0000u);
+            wire[2] = __uint_as_float(w2.y << 16); wire[3] = __uint_as_float(w2.y & 0xFFFF0000u);
+          }
+        } else {
+#pragma unroll
+          for (int x = 0; x < kEpl; ++x) wire[x] = 0.0f;
+        }
+        fence_proxy_async();          // make the shared-memory results visible to the bulk stores
+        __syncwarp();
+        if (lane == 0) mbar_arrive(done_bar(s));
+
+        // ---- drift of the replicas that missed this broadcast ---------------------
+        if constexpr (DRIFTK) {
+          uint64_t sm = stale;
+          while (sm) {
+            // up to four stale copies are fetched before the first is used
+            int ids[4];
+            float old[4][kEpl];
+            int nb = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+              ids[b] = -1;
+              if (sm) {
+                ids[b] = __ffsll((long long)sm) - 1;
+                sm &= sm - 1;
+                nb = b + 1;
+                if (active) {
+                  const typename RT::raw* rp = reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) + e0 + idx;
+                  if constexpr (RT::kVecs == 2) {
+                    const uint4 r = __ldcs(reinterpret_cast<const uint4*>(rp));
+                    old[b][0] = __uint_as_float(r.x); old[b][1] = __uint_as_float(r.y);
+                    old[b][2] = __uint_as_float(r.z); old[b][3] = __uint_as_float(r.w);
+                  } else {
+                    const uint2 r = __ldcs(reinterpret_cast<const uint2*>(rp));
+                    old[b][0] = __uint_as_float(r.x << 16); old[b][1] = __uint_as_float(r.x & 0xFFFF0000u);
+                    old[b][2] = __uint_as_float(r.y << 16); old[b][3] = __uint_as_float(r.y & 0xFFFF0000u);
+                  }
+                } else {
+#pragma unroll
+                  for (int x = 0; x < kEpl; ++x) old[b][x] = 0.0f;
+                }
+              }
+            }
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+              if (b < nb) {
+                float sq = 0.0f;
+#pragma unroll
+                for (int x = 0; x < kEpl; ++x) {
+                  const float d = __fsub_rn(old[b][x], wire[x]);
+                  sq = __fadd_rn(sq, __fmul_rn(d, d));
+                }
+                const float tot = warp_sum(sq);
+                if ((ids[b] & 31) == lane) {
+                  if (ids[b] < 32) dacc0 += (double)tot; else dacc1 += (double)tot;
+                }
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ---- common exit: per-CTA drift partials in fixed order, status word ---------------
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) atomicExch(G.status, 1u);
+  if constexpr (DRIFTK) {
+    double* sh = reinterpret_cast<double*>(stage0);   // stages are idle now
+    if (warp < kConsumerWarps) {
+      sh[warp * kMaxW + lane] = dacc0;
+      sh[warp * kMaxW + lane + 32] = dacc1;
+    }
+    __syncthreads();
+    if (threadIdx.x < kMaxW) {
+      double t = 0.0;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) t += sh[w * kMaxW + threadIdx.x];
+      P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
+    }
+  }
+}
+
+}  // namespace lossy

@@ -153,7 +153,7 @@ def compare_outputs(out, ref, what, with_ghat=True):
 def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None, p_param=None, exact=True):
     """Element-by-element parity of a whole (small) run. Returns the GpuRun for further checks."""
     gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param)
-    orc = make_oracle(w, flags=flags, p_grad=p_grad, p_param=p_param)
+    orc = make_oracle(w, flags=flags & 3, p_grad=p_grad, p_param=p_param)   # bit 4 only picks the kernel
     for t in range(1, steps + 1):
         gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]
         gd = [g.cuda() for g in gs]
@@ -161,6 +161,7 @@ def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None,
         ref = orc.step(t, [to_np(g) for g in gs])
         compare_outputs(gpu.outputs(), ref, f"{w.name} step {t}")
         compare_state(gpu, orc, f"{w.name} step {t}")
+    L.lossy_device_status(gpu.ctx)      # raises if a bounded wait inside a kernel gave up
     if exact:
         # fixed order + separately rounded operations on both sides: the state is in fact bit-identical
         assert_same(to_np(gpu.master), orc.master, f"{w.name} master bits")

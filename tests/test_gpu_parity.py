@@ -10,25 +10,29 @@ from parity_util import (GpuRun, assert_rel, assert_same, compare_outputs, compa
 
 pytestmark = pytest.mark.gpu
 CFG = workload.baseline_workloads()
-LOSSLESS, SKIP = L.LOSSY_SELF_LOSSLESS, L.LOSSY_ZERO_SKIP
+LOSSLESS, SKIP, REG = L.LOSSY_SELF_LOSSLESS, L.LOSSY_ZERO_SKIP, L.LOSSY_REGISTER_PATH
+# the fused call has two kernels: the bulk-copy pipeline (default) and the register path
+PATHS = pytest.mark.parametrize("path_flag", [0, REG], ids=["bulk", "reg"])
 
 
-def test_config1_w4_sgd_fp32_all_steps():
+@PATHS
+def test_config1_w4_sgd_fp32_all_steps(path_flag):
     w = CFG["cfg1_w4_sgd_f32"]
-    run_parity(w, w.steps)
+    run_parity(w, w.steps, flags=path_flag)
 
 
-@pytest.mark.parametrize("fused", [True, False])
-def test_config2_shape_scaled_ragged(fused):
+@pytest.mark.parametrize("mode", ["bulk", "reg", "unfused"])
+def test_config2_shape_scaled_ragged(mode):
     # W=8, bf16 grads, Adam, P=2048: 37 packets + a short one whose length is not a multiple of 8
     w = workload.scaled(CFG["cfg2_w8_layer_adam"], 2048 * 37 + 1003)
-    run_parity(w, 12, fused=fused)
+    run_parity(w, 12, fused=mode != "unfused", flags=REG if mode == "reg" else 0)
 
 
+@PATHS
 @pytest.mark.parametrize("name", ["cfg3_w64_layer_p01", "cfg3_w64_layer_p10"])
-def test_config3_shape_scaled(name):
+def test_config3_shape_scaled(name, path_flag):
     w = workload.scaled(CFG[name], 4096 * 130 + 40)
-    run_parity(w, 6)
+    run_parity(w, 6, flags=path_flag)
 
 
 @pytest.mark.parametrize("P", [256, 1024, 2048, 4096])
@@ -76,6 +80,12 @@ EDGE = [
     ("both_flags_sgd", 2, 128 * 77, 128, 0.6, "sgd", "f32", "f32", LOSSLESS | SKIP),
     ("w64_fp32", 64, 1024 * 20, 1024, 0.05, "sgd", "f32", "f32", 0),
     ("packet_not_multiple_of_chunk", 5, 1000 * 13 + 24, 1000, 0.15, "adam", "bf16", "bf16", 0),
+    ("bulk_short_last_tile", 8, 1032 * 40 + 512, 1032, 0.2, "adam", "bf16", "bf16", 0),
+    ("bulk_three_tiles_per_packet", 12, 2568 * 17 + 96, 2568, 0.25, "adam", "f32", "bf16", 0),
+    ("bulk_w64_heavy_loss", 64, 1024 * 70, 1024, 0.5, "sgd", "bf16", "f32", 0),
+    ("bulk_w17_two_groups", 17, 2048 * 33, 2048, 0.3, "adam", "bf16", "bf16", SKIP),
+    ("bulk_f32_everything", 9, 1024 * 55 + 1000, 1024, 0.1, "adam", "f32", "f32", LOSSLESS),
+    ("bulk_fewer_tiles_than_ctas", 8, 4096 * 3, 4096, 0.3, "adam", "bf16", "bf16", 0),
 ]
 
 
@@ -108,10 +118,12 @@ def test_fused_equals_unfused_bitwise_and_without_optional_outputs():
             assert torch.equal(x.master, y.master) and torch.equal(x.m, y.m) and torch.equal(x.v, y.v)
             for i in range(w.W):
                 assert torch.equal(x.replicas[i], y.replicas[i])
-            assert torch.equal(x.norms, y.norms)
+            # same numbers summed in another fixed order
+            assert torch.allclose(x.norms, y.norms, rtol=2e-6, atol=0)
+        assert torch.equal(a.norms, c.norms)
         assert torch.equal(a.ghat, b.ghat) and torch.equal(a.count, b.count)
         assert torch.equal(a.recv, b.recv) and torch.equal(a.stale, b.stale)
-        assert torch.equal(a.sumsq, b.sumsq)
+        assert torch.allclose(a.sumsq, b.sumsq, rtol=4e-6, atol=0)
 
 
 def test_checkpoint_resume_is_bit_identical():
