@@ -78,13 +78,13 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 }
 
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
-constexpr uint32_t kTmaSmemBudget = 112 * 1024;   // two CTAs per SM
 constexpr uint32_t kTmaSmemFixed = 128 + kMaxStages * sizeof(StageHdr);
 
+template <int CW>
 bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
+  constexpr uint32_t kTile = TmaShape<CW>::kTile;
   const lossy_config& c = ctx->cfg;
-  if (c.flags & LOSSY_REGISTER_PATH) return false;
-  if (c.packet_elems < (uint32_t)kTile) return false;        // small packets: the register kernel
+  if (c.packet_elems < kTile) return false;
   const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
   if (kfull == 0) return false;
   const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
@@ -92,7 +92,7 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   G.groups = (c.W + kGroup - 1) / kGroup;
   uint32_t sb = G.grad_slots * kTile * gb + 3 * kTile * 4 + kTile * rb;
   G.stage_bytes = (sb + 127u) & ~127u;
-  uint32_t budget = kTmaSmemBudget;
+  uint32_t budget = (227u * 1024u) / TmaShape<CW>::kCtasPerSm - 1024u;   // the CTAs of one SM share 227 KB
   if ((uint32_t)ctx->smem_optin < budget) budget = (uint32_t)ctx->smem_optin;
   if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
   G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
@@ -105,20 +105,21 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   return true;
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW>
 int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK>;
+  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW>;
+  constexpr int kThreadsTma = TmaShape<CW>::kThreads;
   const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kTmaThreads, smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreadsTma, smem);
   if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
   if (per_sm < 1) per_sm = 1;
-  if (per_sm > 2) per_sm = 2;
+  if (per_sm > TmaShape<CW>::kCtasPerSm) per_sm = TmaShape<CW>::kCtasPerSm;
   uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
   if (blocks > G.num_tiles) blocks = G.num_tiles;
-  kern<<<blocks, kTmaThreads, smem, s>>>(P, G);
+  kern<<<blocks, kThreadsTma, smem, s>>>(P, G);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda(ctx, "bulk-copy kernel launch", e);
   ctx->launches++;
@@ -126,15 +127,33 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   return LOSSY_OK;
 }
 
-template <bool DRIFTK>
+template <bool DRIFTK, int CW>
 int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
   const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
   const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
   const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
-  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK>(ctx, P, G, s, blocks);
-  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK>(ctx, P, G, s, blocks);
-  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK>(ctx, P, G, s, blocks);
-  return adam ? launch_tma<F32, F32, 1, DRIFTK>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK>(ctx, P, G, s, blocks);
+  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
+  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
+}
+
+// Pick the geometry: wide tiles when a tile has a single worker group and packets are large
+// enough, else the twin-CTA build; false = no bulk-copy launch (register path takes everything).
+int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
+  *used = false;
+  if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
+  TmaGeom G;
+  const bool wide_ok = ctx->cfg.W <= (uint32_t)kGroup && ctx->cfg.packet_elems % TmaShape<16>::kTile == 0;
+  if (wide_ok && tma_geometry<16>(ctx, G)) {
+    *used = true;
+    return drift ? dispatch_tma<true, 16>(ctx, P, G, s, blocks) : dispatch_tma<false, 16>(ctx, P, G, s, blocks);
+  }
+  if (tma_geometry<8>(ctx, G)) {
+    *used = true;
+    return drift ? dispatch_tma<true, 8>(ctx, P, G, s, blocks) : dispatch_tma<false, 8>(ctx, P, G, s, blocks);
+  }
+  return LOSSY_OK;
 }
 
 template <int PH, class GT, class RT, int OPT>
@@ -344,12 +363,12 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, fl
   cudaStream_t s = (cudaStream_t)stream;
   const bool drift = norms || sumsq;
   uint32_t rows = 0;
-  TmaGeom G;
-  if (tma_geometry(ctx, G)) {
-    // complete packets go through the bulk-copy pipeline, a short last packet through the register kernel
-    uint32_t blocks = 0;
-    if (int rc = drift ? dispatch_tma<true>(ctx, P, G, s, &blocks) : dispatch_tma<false>(ctx, P, G, s, &blocks)) return rc;
-    rows = blocks;
+  bool used_tma = false;
+  uint32_t tma_blocks = 0;
+  if (int rc = run_tma(ctx, P, drift, s, &tma_blocks, &used_tma)) return rc;
+  if (used_tma) {
+    // complete packets went through the bulk-copy pipeline; a short last packet takes the register kernel
+    rows = tma_blocks;
     P.chunk_begin = (uint32_t)((ctx->cfg.n / ctx->cfg.packet_elems) * ctx->chunks_per_packet);
     P.partials_row0 = rows;
   }

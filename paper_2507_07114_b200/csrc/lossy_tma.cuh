@@ -1,8 +1,8 @@
 // Fused lossy step as a bulk-copy (TMA) pipeline for sm_100a.
 //
-// One CTA = kConsumerWarps compute warps + 1 producer warp + 1 store warp, two CTAs per SM.
+// One CTA = CW compute warps + 1 producer warp + 1 store warp (see TmaShape for the two builds).
 // The bucket's full packets are cut into tiles of at most kTile contiguous elements inside one
-// packet, so one set of delivery masks covers a tile. Per tile and per group of up to 8 workers
+// packet (kTile = 128 * CW), so one set of delivery masks covers a tile. Per tile and per group of up to 8 workers
 // the producer arms an mbarrier and issues 1-D bulk copies global -> shared memory for the
 // DELIVERED workers' pieces only (dropped packets are never read) and, with the last group, for
 // theta / m / v. Compute warps sum the pieces in ascending worker order from shared memory,
@@ -20,10 +20,16 @@
 
 namespace lossy {
 
-constexpr int kConsumerWarps = 8;
 constexpr int kEpl = 4;                                   // elements per compute lane
-constexpr int kTile = kConsumerWarps * 32 * kEpl;         // 1024 elements
-constexpr int kTmaThreads = (kConsumerWarps + 2) * 32;    // + producer warp + store warp
+// Two geometries are built: "wide" = 16 compute warps, one CTA per SM, tiles of 2048 elements
+// (best when a tile has a single worker group, W <= 8); "twin" = 8 compute warps, two CTAs per
+// SM, tiles of 1024 elements (best when a tile takes several worker groups).
+template <int CW> struct TmaShape {
+  static constexpr int kConsumerWarps = CW;
+  static constexpr int kTile = CW * 32 * kEpl;
+  static constexpr int kThreads = (CW + 2) * 32;          // + producer warp + store warp
+  static constexpr int kCtasPerSm = CW >= 16 ? 1 : 2;
+};
 constexpr int kGroup = 8;                                 // workers per pipeline stage
 constexpr int kMaxStages = 4;
 constexpr uint32_t kMaxPolls = 1u << 22;
@@ -93,34 +99,74 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
-template <class T, int N> struct LaneVec;   // N elements of type T as one shared-memory access
-template <> struct LaneVec<F32, 4> { using type = uint4; };
-template <> struct LaneVec<BF16, 4> { using type = uint2; };
-
+// kEpl consecutive elements of one lane, to and from shared or global memory
 template <class T>
-__device__ __forceinline__ void lds4(const unsigned char* base, uint32_t idx, float (&f)[4]) {
+__device__ __forceinline__ void unpack_lane(const uint32_t (&w)[4], float (&f)[kEpl]) {
   if constexpr (T::kVecs == 2) {
-    const uint4 r = *reinterpret_cast<const uint4*>(base + (size_t)idx * 4);
-    f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y); f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+#pragma unroll
+    for (int x = 0; x < kEpl; ++x) f[x] = __uint_as_float(w[x]);
   } else {
-    const uint2 r = *reinterpret_cast<const uint2*>(base + (size_t)idx * 2);
-    f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xFFFF0000u);
-    f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xFFFF0000u);
+#pragma unroll
+    for (int x = 0; x < kEpl / 2; ++x) {
+      f[2 * x] = __uint_as_float(w[x] << 16);
+      f[2 * x + 1] = __uint_as_float(w[x] & 0xFFFF0000u);
+    }
   }
 }
-__device__ __forceinline__ void sts4_f32(unsigned char* base, uint32_t idx, const float (&f)[4]) {
-  *reinterpret_cast<uint4*>(base + (size_t)idx * 4) =
-      make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+// words of kEpl elements: fp32 -> kEpl words, bf16 -> kEpl/2 words
+template <class T> struct LaneWords { static constexpr int value = T::kVecs == 2 ? kEpl : kEpl / 2; };
+
+template <int WORDS>
+__device__ __forceinline__ void load_words(const void* p, uint32_t (&w)[4]) {
+  if constexpr (WORDS == 4) {
+    const uint4 r = *reinterpret_cast<const uint4*>(p); w[0] = r.x; w[1] = r.y; w[2] = r.z; w[3] = r.w;
+  } else if constexpr (WORDS == 2) {
+    const uint2 r = *reinterpret_cast<const uint2*>(p); w[0] = r.x; w[1] = r.y;
+  } else {
+    w[0] = *reinterpret_cast<const uint32_t*>(p);
+  }
 }
-__device__ __forceinline__ uint2 pack_bf16x4(const float (&f)[4]) {
-  __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]);
-  __nv_bfloat162 b = __floats2bfloat162_rn(f[2], f[3]);
-  return make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+template <int WORDS>
+__device__ __forceinline__ void load_words_stream(const void* p, uint32_t (&w)[4]) {
+  if constexpr (WORDS == 4) {
+    const uint4 r = __ldcs(reinterpret_cast<const uint4*>(p)); w[0] = r.x; w[1] = r.y; w[2] = r.z; w[3] = r.w;
+  } else if constexpr (WORDS == 2) {
+    const uint2 r = __ldcs(reinterpret_cast<const uint2*>(p)); w[0] = r.x; w[1] = r.y;
+  } else {
+    w[0] = __ldcs(reinterpret_cast<const uint32_t*>(p));
+  }
+}
+template <int WORDS>
+__device__ __forceinline__ void store_words(void* p, const uint32_t (&w)[4]) {
+  if constexpr (WORDS == 4) *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+  else if constexpr (WORDS == 2) *reinterpret_cast<uint2*>(p) = make_uint2(w[0], w[1]);
+  else *reinterpret_cast<uint32_t*>(p) = w[0];
+}
+template <class T>
+__device__ __forceinline__ void lds_lane(const unsigned char* base, uint32_t idx, float (&f)[kEpl]) {
+  uint32_t w[4];
+  load_words<LaneWords<T>::value>(base + (size_t)idx * sizeof(typename T::raw), w);
+  unpack_lane<T>(w, f);
+}
+__device__ __forceinline__ void sts_lane_f32(unsigned char* base, uint32_t idx, const float (&f)[kEpl]) {
+  uint32_t w[4];
+#pragma unroll
+  for (int x = 0; x < kEpl; ++x) w[x] = __float_as_uint(f[x]);
+  store_words<kEpl>(base + (size_t)idx * 4, w);
+}
+__device__ __forceinline__ void pack_bf16_lane(const float (&f)[kEpl], uint32_t (&w)[4]) {
+#pragma unroll
+  for (int x = 0; x < kEpl / 2; ++x) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(f[2 * x], f[2 * x + 1]);
+    w[x] = *reinterpret_cast<uint32_t*>(&a);
+  }
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK>
-__global__ void __launch_bounds__(kTmaThreads, 2) lossy_fused_tma_kernel(const __grid_constant__ Params P,
-                                                                         const __grid_constant__ TmaGeom G) {
+template <class GT, class RT, int OPT, bool DRIFTK, int CW>
+__global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPerSm)
+    lossy_fused_tma_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
+  constexpr int kConsumerWarps = CW;
+  constexpr int kTile = TmaShape<CW>::kTile;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
   // layout: [full, done, empty barriers | abort flag] (128 B) | headers (kMaxStages x 64 B) | stages
@@ -265,7 +311,7 @@ __global__ void __launch_bounds__(kTmaThreads, 2) lossy_fused_tma_kernel(const _
           for (int u = 0; u < kGroup; ++u)
             if ((bits >> u) & 1u) {
               float f[kEpl];
-              lds4<GT>(st + (size_t)u * kTile * kGB, idx, f);
+              lds_lane<GT>(st + (size_t)u * kTile * kGB, idx, f);
 #pragma unroll
               for (int x = 0; x < kEpl; ++x) acc[x] = __fadd_rn(acc[x], f[x]);
             }
@@ -285,16 +331,18 @@ __global__ void __launch_bounds__(kTmaThreads, 2) lossy_fused_tma_kernel(const _
 #pragma unroll
             for (int x = 0; x < kEpl; ++x) acc[x] = __fdiv_rn(acc[x], fc);
           }
-          if (P.ghat)
-            __stcs(reinterpret_cast<uint4*>(P.ghat + e0 + idx),
-                   make_uint4(__float_as_uint(acc[0]), __float_as_uint(acc[1]), __float_as_uint(acc[2]),
-                              __float_as_uint(acc[3])));
+          if (P.ghat) {
+            uint32_t gw[4];
+#pragma unroll
+            for (int x = 0; x < kEpl; ++x) gw[x] = __float_as_uint(acc[x]);
+            store_words<kEpl>(P.ghat + e0 + idx, gw);
+          }
           float th[kEpl], m[kEpl], v[kEpl];
-          lds4<F32>(st + off_th, idx, th);
+          lds_lane<F32>(st + off_th, idx, th);
           if (!((P.flags & 2u) && cnt == 0)) {
             if constexpr (OPT == 1) {
-              lds4<F32>(st + off_m, idx, m);
-              lds4<F32>(st + off_v, idx, v);
+              lds_lane<F32>(st + off_m, idx, m);
+              lds_lane<F32>(st + off_v, idx, v);
             }
 #pragma unroll
             for (int x = 0; x < kEpl; ++x) {
@@ -311,21 +359,21 @@ __global__ void __launch_bounds__(kTmaThreads, 2) lossy_fused_tma_kernel(const _
                 v[x] = vn;
               }
             }
-            sts4_f32(st + off_th, idx, th);
+            sts_lane_f32(st + off_th, idx, th);
             if constexpr (OPT == 1) {
-              sts4_f32(st + off_m, idx, m);
-              sts4_f32(st + off_v, idx, v);
+              sts_lane_f32(st + off_m, idx, m);
+              sts_lane_f32(st + off_v, idx, v);
             }
           }
           if constexpr (RT::kVecs == 2) {
-            sts4_f32(st + off_wire, idx, th);
+            sts_lane_f32(st + off_wire, idx, th);
 #pragma unroll
             for (int x = 0; x < kEpl; ++x) wire[x] = th[x];
           } else {
-            const uint2 w2 = pack_bf16x4(th);
-            *reinterpret_cast<uint2*>(st + off_wire + (size_t)idx * 2) = w2;
-            wire[0] = __uint_as_float(w2.x << 16); wire[1] = __uint_as_float(w2.x & 0xFFFF0000u);
-            wire[2] = __uint_as_float(w2.y << 16); wire[3] = __uint_as_float(w2.y & 0xFFFF0000u);
+            uint32_t ww[4];
+            pack_bf16_lane(th, ww);
+            store_words<kEpl / 2>(st + off_wire + (size_t)idx * 2, ww);
+            unpack_lane<BF16>(ww, wire);
           }
         } else {
 #pragma unroll
@@ -352,15 +400,9 @@ __global__ void __launch_bounds__(kTmaThreads, 2) lossy_fused_tma_kernel(const _
                 nb = b + 1;
                 if (active) {
                   const typename RT::raw* rp = reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) + e0 + idx;
-                  if constexpr (RT::kVecs == 2) {
-                    const uint4 r = __ldcs(reinterpret_cast<const uint4*>(rp));
-                    old[b][0] = __uint_as_float(r.x); old[b][1] = __uint_as_float(r.y);
-                    old[b][2] = __uint_as_float(r.z); old[b][3] = __uint_as_float(r.w);
-                  } else {
-                    const uint2 r = __ldcs(reinterpret_cast<const uint2*>(rp));
-                    old[b][0] = __uint_as_float(r.x << 16); old[b][1] = __uint_as_float(r.x & 0xFFFF0000u);
-                    old[b][2] = __uint_as_float(r.y << 16); old[b][3] = __uint_as_float(r.y & 0xFFFF0000u);
-                  }
+                  uint32_t ow[4];
+                  load_words_stream<LaneWords<RT>::value>(rp, ow);
+                  unpack_lane<RT>(ow, old[b]);
                 } else {
 #pragma unroll
                   for (int x = 0; x < kEpl; ++x) old[b][x] = 0.0f;

@@ -1,0 +1,83 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot run a whole 202-million-element bucket in seconds, but packets evolve
+independently: the GPU runs the full bucket, and the oracle re-runs sampled slabs of packets
+(first, last, shard boundaries, random) from regenerated inputs, element by element. The
+drift norms are checked on EVERY element: the oracle's drift routine reads the full GPU
+state copied to the host.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2507_07114_b200 as L
+import workload
+from parity_util import (GpuRun, assert_rel, assert_same, compare_state, make_oracle, to_np)
+
+pytestmark = pytest.mark.gpu
+CFG = workload.baseline_workloads()
+
+
+def _slabs(w, rng, n_random, width):
+    K = w.K
+    pps = (K + w.W - 1) // w.W
+    starts = {0, max(0, K - width), max(0, pps - width // 2), max(0, min(K - width, (w.W - 1) * pps - 1))}
+    starts |= {int(x) for x in rng.integers(0, max(1, K - width), n_random)}
+    return sorted(starts)
+
+
+def _run_full(w, steps, slab_packets, n_random, full_drift):
+    gpu = GpuRun(w)
+    rng = np.random.default_rng(0)
+    slabs = _slabs(w, rng, n_random, slab_packets)
+    P = w.packet_elems
+    oracles = []
+    for k0 in slabs:
+        e0, e1 = k0 * P, min(w.n, (k0 + slab_packets) * P)
+        oracles.append((k0, e0, e1, make_oracle(w, k0=k0, n_slab=e1 - e0, e0=e0)))
+    for t in range(1, steps + 1):
+        gd = [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)]
+        gpu.step_fused(t, gd)                       # the call bench.py times (with every optional output)
+        out = gpu.outputs()
+        for k0, e0, e1, orc in oracles:
+            ref = orc.step(t, [to_np(g[e0:e1]) for g in gd])
+            k1 = k0 + orc.packets
+            what = f"{w.name} step {t} packets [{k0},{k1})"
+            assert_same(out["count"][k0:k1], ref["count"], what + " count")
+            assert_same(out["recv_bits"][k0:k1], ref["recv_bits"], what + " recv_bits")
+            assert_same(out["stale_bits"][k0:k1], ref["stale_bits"], what + " stale_bits")
+            assert_rel(out["ghat"][e0:e1], ref["ghat"], what + " ghat")
+            compare_state(gpu, orc, what, e0, e1)
+        del gd
+    L.lossy_device_status(gpu.ctx)
+    if full_drift:
+        # every element: oracle drift routine on the full GPU state
+        # (a small oracle object is re-pointed at the full arrays; its drift routine only needs
+        # the replica dtype, W and the element count)
+        drift_orc = make_oracle(workload.scaled(w, 8 * w.W, packet_elems=8), theta0=torch.zeros(8 * w.W))
+        drift_orc.n_slab = w.n
+        drift_orc.master = to_np(gpu.master)
+        drift_orc.replicas = [to_np(r) for r in gpu.replicas]
+        want = np.sqrt(drift_orc.drift_sumsq())
+        assert_rel(out["norms"], want, f"{w.name} drift norms over all elements")
+        assert float(want.max()) > 0.0
+    # conservation over the whole bucket: counts are the popcounts of the receive bits
+    pop = np.array([bin(int(b)).count("1") for b in out["recv_bits"][:5000]])
+    assert_same(out["count"][:5000], pop.astype(np.uint8), "count vs popcount")
+    return gpu
+
+
+def test_config2_full_layer_bucket():
+    w = CFG["cfg2_w8_layer_adam"]
+    _run_full(w, steps=3, slab_packets=6, n_random=6, full_drift=True)
+
+
+def test_config3_full_w64_sampled():
+    w = CFG["cfg3_w64_layer_p10"]
+    _run_full(w, steps=2, slab_packets=3, n_random=3, full_drift=False)
+
+
+def test_config5_point_full_size_small_packets_register_path():
+    # P=256 takes the register-path kernel at full size
+    w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.3)
+    _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
