@@ -37,9 +37,10 @@ METRIC = "lossy aggregate+step+broadcast HBM GB/s"
 WORKLOAD = "cfg2_w8_layer_adam"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the fused kernel on the bench
-# workload, from the ncu capture summarised in profiles/ (null until captured).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the fused kernel, from the ncu capture
+# summarised in profiles/fused_step_cfg2_w8_layer.md: 1774.2 MB on a 33,554,432-element cut of the
+# workload, scaled by the elements processed (traffic is proportional to them).
+NCU_TRAFFIC_SMALL_CASE = (1774.2e6, 33554432)
 
 
 def algorithmic_bytes(w: workload.Workload, n: int | None = None) -> float:
@@ -157,6 +158,7 @@ def main():
     ap.add_argument("--p", type=float, default=None, help="override the drop probability")
     ap.add_argument("--workers", type=int, default=0, help="override W")
     ap.add_argument("--packet-elems", type=int, default=0, help="override the packet size")
+    ap.add_argument("--register-path", action="store_true", help="time the register-path kernel, not the bulk-copy pipeline")
     ap.add_argument("--e2e-steps", type=int, default=-1, help="steps of the host-buffer leg (default: min(steps, 10))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-packets", type=int, default=8192)
@@ -181,6 +183,9 @@ def main():
     if args.packet_elems:
         w = workload.scaled(w, w.n, packet_elems=args.packet_elems)
     warmup = max(3, args.warmup)
+    # the stored ncu traffic figure belongs to the unmodified default workload on the default kernel
+    pristine = (args.workload == WORKLOAD and args.p is None and not args.workers and not args.packet_elems
+                and not args.register_path)
 
     if args.impl == "reference":
         if rank != 0:
@@ -215,7 +220,8 @@ def main():
     adam = w.optimizer == "adam"
     ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems, p_grad=w.p, p_param=w.p, seed=w.seed,
                        grad_dtype=gdt, replica_dtype=rdt, optimizer=w.optimizer, lr=w.lr, beta1=w.beta1,
-                       beta2=w.beta2, eps=w.eps, packet_base=w.packet_base)
+                       beta2=w.beta2, eps=w.eps, packet_base=w.packet_base,
+                       flags=L.LOSSY_REGISTER_PATH if args.register_path else 0)
     master = workload.theta0_slab(w, 0, w.n, dev)
     m = torch.zeros_like(master) if adam else None
     v = torch.zeros_like(master) if adam else None
@@ -319,9 +325,12 @@ def main():
                              "two gradient sets alternate" % (B / 1e9),
                        "drift_norm_max_last_step": final_norm_max},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                         "frac": achieved / peak,
+                         "traffic": (NCU_TRAFFIC_SMALL_CASE[0] * w.n / NCU_TRAFFIC_SMALL_CASE[1]
+                                     if pristine else None),
                          "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured"
-                         else peak_src, "kernel": "lossy_fused_tma_kernel (+ W-warp drift finalize)",
+                         else peak_src, "kernel": ("lossy_kernel<AGG|STEP|BCAST|DRIFT>" if args.register_path else "lossy_fused_tma_kernel")
+                         + " (+ W-warp drift finalize)",
                          "avg_launch_ms": avg_launch_ms, "min_launch_ms": min(per_launch_ms)},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
         }
