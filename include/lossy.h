@@ -42,7 +42,8 @@ extern "C" {
 
 typedef struct lossy_ctx lossy_ctx; /* opaque; host object + small device scratch */
 
-enum { LOSSY_OK = 0, LOSSY_EINVAL = 1, LOSSY_ENOMEM = 2, LOSSY_ECUDA = 3, LOSSY_EDEVICE = 4 };
+enum { LOSSY_OK = 0, LOSSY_EINVAL = 1, LOSSY_ENOMEM = 2, LOSSY_ECUDA = 3, LOSSY_EDEVICE = 4,
+       LOSSY_ELIMIT = 5 /* a size is beyond what drift_norms_static supports */ };
 enum { LOSSY_F32 = 0, LOSSY_BF16 = 1 };  /* element types of gradients / replicas */
 enum { LOSSY_SGD = 0, LOSSY_ADAM = 1 };
 enum {
@@ -150,6 +151,44 @@ int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master,
  */
 int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas,
                 float* norms, double* sumsq, void* stream);
+
+/*
+ * drift_norms_static — the same norms as drift_norms for callers that must not
+ * allocate device memory. The paper has no counterpart: this entry point exists
+ * only for the way the library is embedded.
+ *
+ * Some callers cannot call cudaMalloc: a training loop that lives inside a
+ * framework's frozen memory pool, a process that has already committed all of
+ * HBM to its own buffers, a service that bans allocation calls after start-up
+ * because they synchronise the device. lossy_init allocates (the per-block
+ * partial sums of the drift reduction), so such a caller cannot have a context.
+ * This function therefore takes the configuration itself and keeps the partial
+ * sums in a fixed 512 KB array that is part of the library image (held by every
+ * GPU that loads the library, until the process exits). It calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ *   cfg       host pointer; W, n, packet_elems and replica_dtype are used (the
+ *             chunks of the reduction follow the packet grid), the rest is ignored
+ *   master    [n] fp32 device;  replicas: host array of W device pointers, each [n]
+ *   norms     [W] fp32 device, written, or NULL;  sumsq: [W] fp64 device, ADDED to,
+ *             or NULL (at least one of the two)
+ *
+ * Limits: W <= 64 and ceil(n / packet_elems) * ceil(packet_elems / 256) <=
+ * LOSSY_STATIC_MAX_CHUNKS; anything larger returns LOSSY_ELIMIT and launches
+ * nothing. The grid is capped at the 1024 rows of the static array.
+ * First call on a device: looks up the device address of the static array
+ * (cudaGetSymbolAddress, with that device current) and caches it; make that
+ * first call before any stream capture begins.
+ * Sharing: every call in the process uses the same array and finds the last
+ * call's contents in it; each call overwrites every row it later reads, so
+ * nothing needs clearing, but two calls that overlap on the GPU (different
+ * streams, or different host threads without ordering) race on it: serialise
+ * them on one stream or with events.
+ * Results agree with drift_norms up to the rounding of the fixed summation order.
+ */
+#define LOSSY_STATIC_MAX_CHUNKS 0x7FFFFFFFull
+int drift_norms_static(const lossy_config* cfg, const float* master, const void* const* replicas,
+                       float* norms, double* sumsq, void* stream);
 
 /*
  * lossy_fused_step — steps (2), (3), (4) and the drift norms in ONE pass over

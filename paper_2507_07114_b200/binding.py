@@ -14,14 +14,14 @@ import torch
 
 from . import build as _build
 
-LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE = 0, 1, 2, 3, 4
+LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE, LOSSY_ELIMIT = 0, 1, 2, 3, 4, 5
 LOSSY_F32, LOSSY_BF16 = 0, 1
 LOSSY_SGD, LOSSY_ADAM = 0, 1
 LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_aggregate", "lossy_step", "lossy_broadcast",
-    "drift_norms", "lossy_fused_step", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
+    "drift_norms", "drift_norms_static", "lossy_fused_step", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
 
@@ -70,6 +70,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_broadcast.argtypes = [vp, u64, vp, vp, vp, vp]
     lib.drift_norms.restype = C.c_int
     lib.drift_norms.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.drift_norms_static.restype = C.c_int
+    lib.drift_norms_static.argtypes = [C.POINTER(lossy_config), vp, vp, vp, vp, vp]
     lib.lossy_fused_step.restype = C.c_int
     lib.lossy_fused_step.argtypes = [vp, u64] + [vp] * 12
     lib.lossy_fused_step_host.restype = C.c_int
@@ -157,6 +159,19 @@ def lossy_broadcast(ctx, step, master, replicas, stale_bits=None):
 
 def drift_norms(ctx, master, replicas, norms=None, sumsq=None):
     _check(ctx, load_library().drift_norms(ctx, _p(master), _table(replicas), _p(norms), _p(sumsq), _stream()))
+
+
+def drift_norms_static(*, W, n, packet_elems, replica_dtype, master, replicas, norms=None, sumsq=None):
+    """drift_norms for callers that may not allocate device memory (no context; static scratch in the library).
+
+    Raises LossyError with code LOSSY_ELIMIT when a size is beyond the static scratch's limits."""
+    cfg = lossy_config(W, packet_elems, n, 0, 0.0, 0.0, 0, LOSSY_F32, _dt(replica_dtype), LOSSY_SGD, 0,
+                       0.0, 0.0, 0.0, 0.0)
+    rc = load_library().drift_norms_static(C.byref(cfg), _p(master), _table(replicas), _p(norms), _p(sumsq),
+                                           _stream())
+    if rc != LOSSY_OK:
+        raise LossyError(rc, "drift_norms_static: " + {LOSSY_EINVAL: "bad argument", LOSSY_ELIMIT:
+                         "size beyond the static scratch limits", LOSSY_ECUDA: "CUDA error"}.get(rc, "error"))
 
 
 def lossy_fused_step(ctx, step, grads, master, m, v, replicas, ghat=None, count=None, recv_bits=None,

@@ -8,7 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "liblossy_b200.so")
-SOURCES = ["lossy_api.cu"]
+SOURCES = ["lossy_api.cu", "lossy_noalloc.cu"]
 HEADERS = ["lossy_device.cuh", "lossy_kernels.cuh", "lossy_tma.cuh", os.path.join("..", "..", "include", "lossy.h")]
 
 NVCC_FLAGS = [

@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
 
 // Sum the per-block partials of replica blockIdx.x in a fixed order (lane l takes rows l, l+32, ...,
 // then a shuffle tree); add to sumsq, write the norm. One warp per replica.
-__global__ void drift_finalize_kernel(const double* __restrict__ partials, uint32_t nblocks, uint32_t W,
+static __global__ void drift_finalize_kernel(const double* __restrict__ partials, uint32_t nblocks, uint32_t W,
                                       float* norms, double* sumsq) {
   const uint32_t i = blockIdx.x;
   if (i >= W) return;
@@ -276,7 +276,7 @@ __global__ void drift_finalize_kernel(const double* __restrict__ partials, uint3
 }
 
 // Delivery indicators on a dense grid of tuples (host/device agreement check).
-__global__ void mask_grid_kernel(uint64_t seed, uint64_t step, const uint32_t* src, const uint32_t* dst,
+static __global__ void mask_grid_kernel(uint64_t seed, uint64_t step, const uint32_t* src, const uint32_t* dst,
                                  const uint64_t* packet, uint64_t count, uint32_t T, uint8_t* out) {
   const uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= count) return;
