@@ -161,7 +161,7 @@ def main():
     ap.add_argument("--register-path", action="store_true", help="time the register-path kernel, not the bulk-copy pipeline")
     ap.add_argument("--e2e-steps", type=int, default=-1, help="steps of the host-buffer leg (default: min(steps, 10))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-packets", type=int, default=8192)
+    ap.add_argument("--cpu-sample-packets", type=int, default=16384)
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -308,7 +308,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        r = oracle_arm(w, 5, 1, args.cpu_sample_packets)
+        r = oracle_arm(w, 10, 1, args.cpu_sample_packets)
         cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     if rank == 0:

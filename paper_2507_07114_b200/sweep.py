@@ -1,0 +1,97 @@
+"""Throughput and drift of the fused step over the benchmark configurations.
+
+    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,5] [--steps N]
+
+Prints one line per point: algorithmic GB/s, fraction of the measured HBM copy peak, steps/s and the
+largest per-replica drift norm seen. Inputs are the seeded synthetic workloads; state stays in HBM.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import torch
+
+import workload
+from . import binding as L
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
+def algorithmic_bytes(w):
+    gb = 2 if w.grad_dtype == "bf16" else 4
+    rb = 2 if w.replica_dtype == "bf16" else 4
+    return (1.0 - w.p) * w.W * w.n * gb + (24 if w.optimizer == "adam" else 8) * w.n + w.W * w.n * rb
+
+
+def run_point(w, steps, warmup=3, grad_sets=2):
+    dev = torch.device("cuda")
+    gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    rdt = torch.bfloat16 if w.replica_dtype == "bf16" else torch.float32
+    adam = w.optimizer == "adam"
+    ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems, p_grad=w.p, p_param=w.p, seed=w.seed,
+                       grad_dtype=gdt, replica_dtype=rdt, optimizer=w.optimizer, lr=w.lr, beta1=w.beta1,
+                       beta2=w.beta2, eps=w.eps)
+    master = workload.theta0_slab(w, 0, w.n, dev)
+    m = torch.zeros_like(master) if adam else None
+    v = torch.zeros_like(master) if adam else None
+    reps = [master.to(rdt) for _ in range(w.W)]
+    norms = torch.zeros(w.W, device=dev)
+    worst = torch.zeros(w.W, device=dev)
+    sets = [[workload.grad_slab(w, s, i, 0, w.n, dev) for i in range(w.W)] for s in range(1, grad_sets + 1)]
+    t = 0
+    for _ in range(warmup):
+        t += 1
+        L.lossy_fused_step(ctx, t, sets[t % grad_sets], master, m, v, reps, norms=norms)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        t += 1
+        L.lossy_fused_step(ctx, t, sets[t % grad_sets], master, m, v, reps, norms=norms)
+        torch.maximum(worst, norms, out=worst)
+    e1.record()
+    torch.cuda.synchronize()
+    L.lossy_device_status(ctx)
+    ms = e0.elapsed_time(e1) / steps
+    L.lossy_destroy(ctx)
+    gbs = algorithmic_bytes(w) / (ms * 1e-3) / 1e9
+    return {"workload": w.name, "W": w.W, "P": w.packet_elems, "p": w.p, "ms_per_step": ms, "GBps": gbs,
+            "frac_of_measured_peak": gbs / _peak(), "steps_per_s": 1e3 / ms, "max_drift_norm": float(worst.max())}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--configs", default="1,2,3,5")
+    ap.add_argument("--steps", type=int, default=0, help="0 = each configuration's own step count")
+    args = ap.parse_args()
+    cfg = workload.baseline_workloads()
+    want = set(args.configs.split(","))
+    points = []
+    if "1" in want:
+        points.append(cfg["cfg1_w4_sgd_f32"])
+    if "2" in want:
+        points.append(cfg["cfg2_w8_layer_adam"])
+    if "3" in want:
+        points += [cfg["cfg3_w64_layer_p01"], cfg["cfg3_w64_layer_p10"]]
+    if "5" in want:
+        for P in (256, 1024, 2048, 4096):
+            for p in (0.0, 0.01, 0.05, 0.1, 0.3):
+                points.append(workload.scaled(cfg["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=P, p=p,
+                                              name=f"cfg5_w16_P{P}_p{p}"))
+    for w in points:
+        r = run_point(w, args.steps or w.steps, grad_sets=1 if w.W >= 64 else 2)
+        print(json.dumps(r), flush=True)
+
+
+if __name__ == "__main__":
+    main()
