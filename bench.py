@@ -209,7 +209,7 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or "WORLD_SIZE" in os.environ:         # under torchrun, also with a single rank
         import torch.distributed as dist
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
@@ -308,7 +308,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        r = oracle_arm(w, 10, 1, args.cpu_sample_packets)
+        r = oracle_arm(w, 20, 1, args.cpu_sample_packets)
         cpu = {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     if rank == 0:

@@ -22,8 +22,8 @@ namespace lossy {
 
 constexpr int kEpl = 4;                                   // elements per compute lane
 // Two geometries are built: "wide" = 16 compute warps, one CTA per SM, tiles of 2048 elements
-// (best when a tile has a single worker group, W <= 8); "twin" = 8 compute warps, two CTAs per
-// SM, tiles of 1024 elements (best when a tile takes several worker groups).
+// (best when a tile takes one or two worker groups, W <= 16); "twin" = 8 compute warps, two CTAs
+// per SM, tiles of 1024 elements (best when a tile takes many worker groups).
 template <int CW> struct TmaShape {
   static constexpr int kConsumerWarps = CW;
   static constexpr int kTile = CW * 32 * kEpl;
@@ -41,6 +41,7 @@ struct TmaGeom {
   uint32_t stage_bytes;       // per stage, 128-byte multiple
   uint32_t groups;            // ceil(W / kGroup)
   uint32_t grad_slots;        // min(W, kGroup)
+  uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores
   uint32_t* status;           // device status word (0 = fine)
 };
 
@@ -73,13 +74,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
 }
-__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+// `hint` = mark the lines evict-first in L2 (they are touched once per step)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, bool hint,
+                                         uint64_t pol) {
+  if (hint)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+                 : "memory");
+  else
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void* dst, uint32_t src, uint32_t bytes, bool hint, uint64_t pol) {
+  if (hint)
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(dst), "r"(src),
+                 "r"(bytes), "l"(pol)
+                 : "memory");
+  else
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -203,6 +221,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     // =============================== producer warp ===============================
     uint32_t it = 0, armed_mask = 0, armed_par = 0;
     bool ok = true;
+    const bool lh = G.hints & 1u;
+    const uint64_t pol = policy_evict_first();
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
       const uint32_t k = tile / G.tiles_per_packet;
       const uint32_t c = tile - k * G.tiles_per_packet;
@@ -238,12 +258,12 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         __syncwarp();
         if (lane < kGroup && ((bits >> lane) & 1u))
           bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
-                   reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s));
+                   reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
         if (last) {
-          if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s));
+          if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
           if constexpr (OPT == 1) {
-            if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s));
-            if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s));
+            if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s), lh, pol);
+            if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s), lh, pol);
           }
         }
         armed_mask |= 1u << s;
@@ -261,6 +281,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     // ================================ store warp =================================
     uint32_t it = 0;
     bool ok = true;
+    const bool sh_hint = G.hints & 2u;
+    const uint64_t pol = policy_evict_first();
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
       for (uint32_t g = 0; g < G.groups; ++g, ++it) {
         const uint32_t s = it % S, par = (it / S) & 1u;
@@ -270,14 +292,14 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           const uint64_t e0 = h.e0, stale = h.stale;
           const uint32_t len = h.len;
           unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
-          if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u);
+          if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u, sh_hint, pol);
           if constexpr (OPT == 1) {
-            if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u);
-            if (lane == 2) bulk_s2g(P.v + e0, smem_u32(st + off_v), len * 4u);
+            if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u, sh_hint, pol);
+            if (lane == 2) bulk_s2g(P.v + e0, smem_u32(st + off_v), len * 4u, sh_hint, pol);
           }
           for (uint32_t i = lane; i < W; i += 32)
             if (!((stale >> i) & 1ull))
-              bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB);
+              bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB, sh_hint, pol);
           bulk_commit();
           bulk_wait_read0();          // shared memory of this stage may be overwritten after this
         }

@@ -52,6 +52,7 @@ def run_point(w, steps, warmup=3, grad_sets=2):
     for _ in range(warmup):
         t += 1
         L.lossy_fused_step(ctx, t, sets[t % grad_sets], master, m, v, reps, norms=norms)
+        torch.maximum(worst, norms, out=worst)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
