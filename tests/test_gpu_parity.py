@@ -86,6 +86,12 @@ EDGE = [
     ("bulk_w17_two_groups", 17, 2048 * 33, 2048, 0.3, "adam", "bf16", "bf16", SKIP),
     ("bulk_f32_everything", 9, 1024 * 55 + 1000, 1024, 0.1, "adam", "f32", "f32", LOSSLESS),
     ("bulk_fewer_tiles_than_ctas", 8, 4096 * 3, 4096, 0.3, "adam", "bf16", "bf16", 0),
+    # small packets: a tile of the bulk-copy kernel packs several whole packets
+    ("bulk_packed_256_w16_last_tile_short", 16, 256 * 37 + 100, 256, 0.2, "adam", "bf16", "bf16", 0),
+    ("bulk_packed_128_w40", 40, 128 * 50 + 8, 128, 0.3, "sgd", "bf16", "bf16", 0),
+    ("bulk_packed_512_w3_f32", 3, 512 * 21, 512, 0.4, "adam", "f32", "f32", SKIP),
+    ("bulk_packed_1024_w16", 16, 1024 * 9 + 512, 1024, 0.1, "adam", "bf16", "bf16", LOSSLESS),
+    ("bulk_packed_256_heavy_loss", 8, 256 * 64, 256, 0.6, "adam", "bf16", "bf16", 0),
 ]
 
 
