@@ -54,9 +54,8 @@ enum {
   /* A packet that received nothing leaves theta, m, v untouched. Default: the
    * estimate is exactly 0 and is fed to the unmodified optimizer. */
   LOSSY_ZERO_SKIP = 2u,
-  /* lossy_fused_step always uses the register-path kernel. Default: complete packets go through
-   * the bulk-copy (TMA) pipeline when the packet size is at least 1024 elements, or divides the
-   * tile (128 ... 1024 elements, a multiple of 128). Both kernels give the same state. */
+  /* lossy_fused_step always uses the register-path kernel. Default: complete packets of at
+   * least 1024 elements go through the bulk-copy (TMA) pipeline. Both give the same state. */
   LOSSY_REGISTER_PATH = 4u
 };
 

@@ -88,15 +88,9 @@ template <int CW>
 bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   constexpr uint32_t kTile = TmaShape<CW>::kTile;
   const lossy_config& c = ctx->cfg;
+  if (c.packet_elems < kTile) return false;
   const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
-  if (kfull == 0 || kfull >= (1ull << 31)) return false;
-  G.packets_per_tile = 1;
-  if (c.packet_elems < kTile) {
-    // small packets: a tile packs several whole packets (each compute warp's 128 elements stay in one)
-    if (kTile % c.packet_elems != 0 || c.packet_elems % 128 != 0 || kTile / c.packet_elems > (uint32_t)kMaxSub) return false;
-    G.packets_per_tile = kTile / c.packet_elems;
-  }
-  G.full_packets = (uint32_t)kfull;
+  if (kfull == 0) return false;
   const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
   G.grad_slots = c.W < (uint32_t)kGroup ? c.W : (uint32_t)kGroup;
   G.groups = (c.W + kGroup - 1) / kGroup;
@@ -107,9 +101,8 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
   G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
   if (G.stages > (uint32_t)kMaxStages) G.stages = kMaxStages;
-  G.tiles_per_packet = G.packets_per_tile > 1 ? 1u : (c.packet_elems + kTile - 1) / kTile;
-  const uint64_t tiles = G.packets_per_tile > 1 ? (kfull + G.packets_per_tile - 1) / G.packets_per_tile
-                                                : kfull * G.tiles_per_packet;
+  G.tiles_per_packet = (c.packet_elems + kTile - 1) / kTile;
+  const uint64_t tiles = kfull * G.tiles_per_packet;
   if (tiles >= (1ull << 31)) return false;
   G.num_tiles = (uint32_t)tiles;
   G.status = ctx->status;
@@ -156,8 +149,7 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   *used = false;
   if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
   TmaGeom G;
-  const uint32_t Pk = ctx->cfg.packet_elems, wide_tile = TmaShape<16>::kTile;
-  const bool wide_ok = ctx->cfg.W <= 2u * kGroup && (Pk % wide_tile == 0 || (Pk >= 256 && wide_tile % Pk == 0));
+  const bool wide_ok = ctx->cfg.W <= 2u * kGroup && ctx->cfg.packet_elems % TmaShape<16>::kTile == 0;
   if (wide_ok && tma_geometry<16>(ctx, G)) {
     *used = true;
     return drift ? dispatch_tma<true, 16>(ctx, P, G, s, blocks) : dispatch_tma<false, 16>(ctx, P, G, s, blocks);

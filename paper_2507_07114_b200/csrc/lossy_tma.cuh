@@ -34,13 +34,9 @@ constexpr int kGroup = 8;                                 // workers per pipelin
 constexpr int kMaxStages = 4;
 constexpr uint32_t kMaxPolls = 1u << 22;
 
-constexpr int kMaxSub = 8;                                // packets per tile when packets are small
-
 struct TmaGeom {
-  uint32_t num_tiles;         // large packets: full packets * tiles_per_packet; small: ceil(full / packets_per_tile)
-  uint32_t tiles_per_packet;  // >= 1 when a packet is cut into tiles (packets_per_tile == 1)
-  uint32_t packets_per_tile;  // > 1 when a tile packs several whole packets (tiles_per_packet == 1)
-  uint32_t full_packets;      // packets that are complete (the ragged last one is not ours)
+  uint32_t num_tiles;         // full packets * tiles_per_packet
+  uint32_t tiles_per_packet;
   uint32_t stages;
   uint32_t stage_bytes;       // per stage, 128-byte multiple
   uint32_t groups;            // ceil(W / kGroup)
@@ -49,19 +45,12 @@ struct TmaGeom {
   uint32_t* status;           // device status word (0 = fine)
 };
 
-// What the producer tells the other warps about a stage: the tile's place in the bucket and the
-// delivery masks of each packet (or packet piece) in it.
 struct __align__(16) StageHdr {
-  uint64_t recv[kMaxSub], stale[kMaxSub];
-  uint64_t e0;          // first element of the tile
-  uint32_t len;         // elements in the tile
-  uint32_t npk;         // sub-packets in the tile (1 unless the tile packs small packets)
-  uint32_t sub_len;     // elements per sub-packet
-  uint32_t last;        // this stage carries theta/m/v (last worker group of the tile)
-  uint8_t cnt[kMaxSub];
-  uint32_t pad[22];
+  uint64_t recv, stale, e0;
+  uint32_t k, len, cnt, last;
+  uint32_t pad[6];
 };
-static_assert(sizeof(StageHdr) == 256, "header is one 256-byte slot");
+static_assert(sizeof(StageHdr) == 64, "header is one 64-byte slot");
 
 // ---- PTX wrappers ---------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -198,7 +187,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   constexpr int kTile = TmaShape<CW>::kTile;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
-  // layout: [full, done, empty barriers | abort flag] (128 B) | headers (kMaxStages x 256 B) | stages
+  // layout: [full, done, empty barriers | abort flag] (128 B) | headers (kMaxStages x 64 B) | stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 96);
   StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + 128);
@@ -235,78 +224,41 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     const bool lh = G.hints & 1u;
     const uint64_t pol = policy_evict_first();
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
-      // place of the tile: a piece of one large packet, or up to kMaxSub whole small packets
-      uint32_t k0, npk, sub_len, len;
-      uint64_t e0;
-      bool first_piece;
-      if (G.packets_per_tile > 1) {
-        k0 = tile * G.packets_per_tile;
-        npk = min(G.packets_per_tile, G.full_packets - k0);
-        sub_len = P.P;
-        len = npk * sub_len;
-        e0 = (uint64_t)k0 * P.P;
-        first_piece = true;
-      } else {
-        k0 = tile / G.tiles_per_packet;
-        const uint32_t c = tile - k0 * G.tiles_per_packet;
-        npk = 1;
-        len = min((uint32_t)kTile, P.P - c * kTile);
-        sub_len = len;
-        e0 = (uint64_t)k0 * P.P + (uint64_t)c * kTile;
-        first_piece = c == 0;
+      const uint32_t k = tile / G.tiles_per_packet;
+      const uint32_t c = tile - k * G.tiles_per_packet;
+      const uint32_t j = k / P.pps;
+      const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
+      const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
+      uint64_t recv = 0, stale = 0;
+      packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale);
+      const uint32_t cnt = __popcll(recv);
+      if (c == 0 && lane == 0) {
+        if (P.count) P.count[k] = (uint8_t)cnt;
+        if (P.recv_bits) P.recv_bits[k] = recv;
+        if (P.stale_bits) P.stale_bits[k] = stale;
       }
-      uint64_t recv[kMaxSub], stale[kMaxSub];
-#pragma unroll
-      for (int sp = 0; sp < kMaxSub; ++sp) {
-        recv[sp] = 0; stale[sp] = 0;
-        if ((uint32_t)sp < npk) {
-          const uint32_t k = k0 + sp;
-          packet_masks<AGG | BCAST>(P, k, k / P.pps, lane, recv[sp], stale[sp]);
-          if (first_piece && lane == 0) {
-            if (P.count) P.count[k] = (uint8_t)__popcll(recv[sp]);
-            if (P.recv_bits) P.recv_bits[k] = recv[sp];
-            if (P.stale_bits) P.stale_bits[k] = stale[sp];
-          }
-          if constexpr (DRIFTK) {
-            for (uint32_t i = lane; i < W; i += 32)
-              if ((stale[sp] >> i) & 1ull)
-                bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0 + (uint64_t)sp * sub_len,
-                                 sub_len * kRB);
-          }
-        }
+      if constexpr (DRIFTK) {
+        for (uint32_t i = lane; i < W; i += 32)
+          if ((stale >> i) & 1ull)
+            bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
       }
       for (uint32_t g = 0; g < G.groups; ++g, ++it) {
         const uint32_t s = it % S, par = (it / S) & 1u;
         if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
         const bool last = g + 1 == G.groups;
+        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & 0xFFu;
         unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
         if (lane == 0) {
           StageHdr& h = hdrs[s];
-          uint32_t delivered = 0;
-#pragma unroll
-          for (int sp = 0; sp < kMaxSub; ++sp) {
-            h.recv[sp] = recv[sp]; h.stale[sp] = stale[sp]; h.cnt[sp] = (uint8_t)__popcll(recv[sp]);
-            delivered += __popc((uint32_t)(recv[sp] >> (g * kGroup)) & 0xFFu);
-          }
-          h.e0 = e0; h.len = len; h.npk = npk; h.sub_len = sub_len; h.last = last ? 1u : 0u;
-          uint32_t bytes = delivered * sub_len * kGB;
+          h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
+          uint32_t bytes = __popc(bits) * len * kGB;
           if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
           mbar_arrive_expect_tx(full_bar(s), bytes);
         }
         __syncwarp();
-        // one bulk copy per delivered (sub-packet, worker of this group) pair, spread over the lanes
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint32_t pair = lane + 32 * half;     // pair = sp * kGroup + u
-          const uint32_t sp = pair / kGroup, u = pair % kGroup;
-          uint64_t r = 0;
-#pragma unroll
-          for (int q = 0; q < kMaxSub; ++q) r = (uint32_t)q == sp ? recv[q] : r;
-          if (sp < npk && ((r >> (g * kGroup + u)) & 1ull))
-            bulk_g2s(smem_u32(st + ((size_t)u * kTile + (size_t)sp * sub_len) * kGB),
-                     reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + u]) + e0 + (uint64_t)sp * sub_len,
-                     sub_len * kGB, full_bar(s), lh, pol);
-        }
+        if (lane < kGroup && ((bits >> lane) & 1u))
+          bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
+                   reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
         if (last) {
           if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
           if constexpr (OPT == 1) {
@@ -337,29 +289,17 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         if (!mbar_wait(done_bar(s), par, abort_flag)) { ok = false; break; }
         if (g + 1 == G.groups) {
           const StageHdr& h = hdrs[s];
-          const uint64_t e0 = h.e0;
-          const uint32_t len = h.len, npk = h.npk, sub_len = h.sub_len;
+          const uint64_t e0 = h.e0, stale = h.stale;
+          const uint32_t len = h.len;
           unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
           if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u, sh_hint, pol);
           if constexpr (OPT == 1) {
             if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u, sh_hint, pol);
             if (lane == 2) bulk_s2g(P.v + e0, smem_u32(st + off_v), len * 4u, sh_hint, pol);
           }
-          // replica i takes every run of consecutive sub-packets whose broadcast it received
-          for (uint32_t i = lane; i < W; i += 32) {
-            int run = -1;
-#pragma unroll
-            for (int sp = 0; sp <= kMaxSub; ++sp) {
-              const bool fresh = sp < kMaxSub && (uint32_t)sp < npk && !((h.stale[sp < kMaxSub ? sp : 0] >> i) & 1ull);
-              if (fresh && run < 0) run = sp;
-              if (!fresh && run >= 0) {
-                bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0 + (uint64_t)run * sub_len,
-                         smem_u32(st + off_wire + (size_t)run * sub_len * kRB), (uint32_t)(sp - run) * sub_len * kRB,
-                         sh_hint, pol);
-                run = -1;
-              }
-            }
-          }
+          for (uint32_t i = lane; i < W; i += 32)
+            if (!((stale >> i) & 1ull))
+              bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB, sh_hint, pol);
           bulk_commit();
           bulk_wait_read0();          // shared memory of this stage may be overwritten after this
         }
@@ -379,13 +319,9 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint32_t s = it % S, par = (it / S) & 1u;
         if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
         const StageHdr& h = hdrs[s];
+        const uint64_t recv = h.recv;
         const uint32_t len = h.len;
         const bool active = idx < len;
-        // the 128 elements of this warp lie inside one sub-packet (its length is a multiple of 128)
-        const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;   // first element of this warp
-        const bool warp_active = widx < len;
-        const uint32_t sp = (h.npk > 1 && warp_active) ? widx / h.sub_len : 0u;
-        const uint64_t recv = h.recv[sp];
         unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
         if (g == 0) {
 #pragma unroll
@@ -408,8 +344,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           continue;
         }
         // ---- last group of the tile: estimate, update, wire value -----------------
-        const uint32_t cnt = h.cnt[sp];
-        const uint64_t stale = warp_active ? h.stale[sp] : 0ull, e0 = h.e0;   // warp-uniform
+        const uint32_t cnt = h.cnt;
+        const uint64_t stale = h.stale, e0 = h.e0;
         float wire[kEpl];
         if (active) {
           if (cnt > 0) {
