@@ -66,6 +66,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   P.Tg = ctx->Tg;
   P.Tp = ctx->Tp;
   P.flags = c.flags;
+  P.prefetch_next = c.W <= 8u ? 1u : 0u;
   P.lr = c.lr;
   P.b1 = c.beta1;
   P.b2 = c.beta2;

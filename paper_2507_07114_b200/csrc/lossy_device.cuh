@@ -50,6 +50,7 @@ struct Params {
   uint32_t W;
   uint32_t Tg, Tp;        // drop iff hash < T
   uint32_t flags;
+  uint32_t prefetch_next; // register kernel: L2-prefetch the warp's next chunk
   float lr, b1, b2, omb1, omb2, ibc1, ibc2, eps;
 };
 
