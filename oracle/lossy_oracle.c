@@ -120,8 +120,13 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
  *   grads[i]        worker i's gradient slab (cfg.grad_dtype), read only
  *   master, m, v    REAL [n_slab], updated in place (m, v ignored for SGD)
  *   replicas[i]     worker i's copy of the slab (cfg.replica_dtype), updated in place
+ *   ghat_prev       NULL: Section 3's per-link loss (the default). Non-NULL (REAL [n_slab], in/out):
+ *                   Algorithm 1's gradient half — the reduce over all W workers is reliable,
+ *                   then ONE draw per packet decides whether the owner keeps the fresh aggregate
+ *                   (and saves it as "prev") or falls back to the saved previous aggregate
  *   recv_force      optional [packets] uint64: use these delivery bits (bit i = s_i)
  *                   instead of the hash — the hook the exhaustive-pattern test uses
+ *                   (Algorithm 1 mode: bit 0 = the packet's aggregate survives)
  *   stale_force     optional [packets] uint64: bit i = replica i misses the broadcast
  *   ghat            optional REAL [n_slab] out
  *   count           optional uint8 [packets] out; recv_bits / stale_bits optional uint64 [packets] out
@@ -131,7 +136,7 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
  */
 int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_slab,
                const void* const* grads, REAL* master, REAL* m, REAL* v, void* const* replicas,
-               const uint64_t* recv_force, const uint64_t* stale_force,
+               REAL* ghat_prev, const uint64_t* recv_force, const uint64_t* stale_force,
                REAL* ghat, uint8_t* count, uint64_t* recv_bits, uint64_t* stale_bits,
                uint32_t* const* age, double* sumsq) {
   if (!c || c->W == 0 || c->W > 64 || c->packet_elems == 0) return 1;
@@ -158,7 +163,11 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
 
     /* (2) which workers' pieces reached the owner: s^(i,j) */
     uint64_t recv = 0;
-    if (recv_force) recv = recv_force[kl];
+    if (ghat_prev) {
+      /* Algorithm 1: "reduce-scatter" is lossless, then Uniform(0,1) < p_grad drops the whole packet */
+      int keep = recv_force ? (int)(recv_force[kl] & 1ULL) : (NAME(hash_u32)(c->seed, step, j, j, kg) >= Tg);
+      if (keep) recv = W == 64 ? ~0ULL : ((1ULL << W) - 1ULL);
+    } else if (recv_force) recv = recv_force[kl];
     else
       for (uint32_t i = 0; i < W; ++i) {
         int s = NAME(hash_u32)(c->seed, step, i, j, kg) >= Tg;
@@ -184,6 +193,11 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
       for (uint32_t i = 0; i < W; ++i)
         if ((recv >> i) & 1ULL) acc = acc + load_grad(grads[i], c->grad_dtype, e);
       REAL gh = cnt > 0 ? acc / (REAL)cnt : (REAL)0;
+      if (ghat_prev) {
+        /* Algorithm 1: dropped => g <- g_prev ; else g_prev <- g */
+        if (cnt == 0) gh = ghat_prev[e];
+        else ghat_prev[e] = gh;
+      }
       if (ghat) ghat[e] = gh;
 
       /* (3) the owner's update of its shard */

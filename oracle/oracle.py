@@ -78,7 +78,7 @@ def _lib(f64: bool):
         o.argtypes = [C.POINTER(OracleConfig), C.c_uint64]
         s = getattr(lib, pre + "step")
         s.restype = C.c_int
-        s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 13
+        s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 14
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
         ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -131,7 +131,7 @@ class Oracle:
 
     def __init__(self, *, W, n, packet_elems, p_grad, p_param, seed, grad_dtype, replica_dtype,
                  optimizer, theta0, lr, beta1=0.9, beta2=0.95, eps=1e-8, flags=0, packet_base=0,
-                 k0=0, n_slab=None, f64=False, track_age=False):
+                 k0=0, n_slab=None, f64=False, track_age=False, alg1=False):
         self.cfg = OracleConfig(W, packet_elems, n, packet_base, p_grad, p_param, seed, grad_dtype,
                                 replica_dtype, optimizer, flags, lr, beta1, beta2, eps)
         self.W, self.P, self.n, self.k0 = W, packet_elems, n, k0
@@ -148,6 +148,8 @@ class Oracle:
         wire = cast_wire(theta0, replica_dtype)
         self.replicas = [wire.copy() for _ in range(W)]
         self.age = [np.zeros(self.packets, np.uint32) for _ in range(W)] if track_age else None
+        # Algorithm 1's gradient half keeps the last surviving aggregate per element ("g_prev"), zero at start
+        self.ghat_prev = np.zeros(self.n_slab, self.real) if alg1 else None
         self.grad_dtype, self.replica_dtype = grad_dtype, replica_dtype
 
     def owner(self, k: int) -> int:
@@ -174,7 +176,8 @@ class Oracle:
             stale_force = np.ascontiguousarray(stale_force, dtype=np.uint64)
         rc = getattr(self.lib, self.pre + "step")(
             C.byref(self.cfg), t, self.k0, self.n_slab, C.cast(gt, C.c_void_p), _ptr(self.master),
-            _ptr(self.m), _ptr(self.v), C.cast(rt, C.c_void_p), _ptr(recv_force), _ptr(stale_force),
+            _ptr(self.m), _ptr(self.v), C.cast(rt, C.c_void_p), _ptr(self.ghat_prev), _ptr(recv_force),
+            _ptr(stale_force),
             _ptr(ghat), _ptr(count), _ptr(recv), _ptr(stale),
             C.cast(at, C.c_void_p) if at is not None else None, _ptr(sumsq))
         if rc != 0:
