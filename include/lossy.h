@@ -206,6 +206,31 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads,
                      uint64_t* stale_bits, float* norms, double* sumsq, void* stream);
 
 /*
+ * lossy_aggregate_alg1 / lossy_fused_step_alg1 — the gradient half of the paper's
+ * Algorithm 1 ("Drop simulation on worker n") in place of Section 3's per-link loss:
+ * the gradient reduce is reliable (plain mean over all W workers, ascending order,
+ * fp32, divided by W), then ONE draw per packet,
+ *     keep = hash(seed, step, src=owner, dst=owner, packet_base+k) >= T_grad,
+ * decides: keep => ghat = mean and ghat_prev <- mean; drop => ghat = ghat_prev and
+ * ghat_prev is left as it was (Algorithm 1: "drop gradient: g <- g_prev, else
+ * g_prev <- g"). "Renormalise surviving shards" is read as the division of the
+ * reduced sum by the worker count. Shard-granular loss, as the algorithm prints it,
+ * is packet_elems = shard length. The parameter half (stale-retaining broadcast with
+ * p_param) and everything else are those of lossy_aggregate / lossy_fused_step.
+ *   ghat_prev  [n] fp32 device, caller-owned state, zero before the first step;
+ *              read on a drop, written on a keep
+ *   count[k]   W for a kept packet, 0 for a dropped one; recv_bits all ones / zero
+ * Gradients of a dropped packet are not read. LOSSY_SELF_LOSSLESS contexts are
+ * rejected (LOSSY_EINVAL); with LOSSY_ZERO_SKIP a dropped packet skips the optimizer.
+ */
+int lossy_aggregate_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev,
+                         float* ghat, uint8_t* count, uint64_t* recv_bits, void* stream);
+int lossy_fused_step_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev,
+                          float* master, float* m, float* v, void* const* replicas,
+                          float* ghat, uint8_t* count, uint64_t* recv_bits,
+                          uint64_t* stale_bits, float* norms, double* sumsq, void* stream);
+
+/*
  * lossy_fused_step_host — the same step for a caller whose gradients live in
  * HOST memory (pinned memory for full copy speed): copies worker i's gradient
  * from host_grads[i] into dev_grads[i] on `stream`, runs lossy_fused_step, and

@@ -21,7 +21,7 @@ LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_aggregate", "lossy_step", "lossy_broadcast",
-    "drift_norms", "drift_norms_static", "lossy_fused_step", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
+    "drift_norms", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
 
@@ -74,6 +74,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.drift_norms_static.argtypes = [C.POINTER(lossy_config), vp, vp, vp, vp, vp]
     lib.lossy_fused_step.restype = C.c_int
     lib.lossy_fused_step.argtypes = [vp, u64] + [vp] * 12
+    lib.lossy_aggregate_alg1.restype = C.c_int
+    lib.lossy_aggregate_alg1.argtypes = [vp, u64, vp, vp, vp, vp, vp, vp]
+    lib.lossy_fused_step_alg1.restype = C.c_int
+    lib.lossy_fused_step_alg1.argtypes = [vp, u64] + [vp] * 13
     lib.lossy_fused_step_host.restype = C.c_int
     lib.lossy_fused_step_host.argtypes = [vp, u64] + [vp] * 9
     lib.lossy_mask.restype = C.c_int
@@ -179,6 +183,18 @@ def lossy_fused_step(ctx, step, grads, master, m, v, replicas, ghat=None, count=
     _check(ctx, load_library().lossy_fused_step(ctx, step, _table(grads), _p(master), _p(m), _p(v), _table(replicas),
                                                 _p(ghat), _p(count), _p(recv_bits), _p(stale_bits), _p(norms),
                                                 _p(sumsq), _stream()))
+
+
+def lossy_aggregate_alg1(ctx, step, grads, ghat_prev, ghat, count=None, recv_bits=None):
+    _check(ctx, load_library().lossy_aggregate_alg1(ctx, step, _table(grads), _p(ghat_prev), _p(ghat), _p(count),
+                                                    _p(recv_bits), _stream()))
+
+
+def lossy_fused_step_alg1(ctx, step, grads, ghat_prev, master, m, v, replicas, ghat=None, count=None,
+                          recv_bits=None, stale_bits=None, norms=None, sumsq=None):
+    _check(ctx, load_library().lossy_fused_step_alg1(ctx, step, _table(grads), _p(ghat_prev), _p(master), _p(m),
+                                                     _p(v), _table(replicas), _p(ghat), _p(count), _p(recv_bits),
+                                                     _p(stale_bits), _p(norms), _p(sumsq), _stream()))
 
 
 def lossy_fused_step_host(ctx, step, host_grads, dev_grads, master, m, v, replicas, dev_norms, host_norms):

@@ -266,9 +266,8 @@ int lossy_set_lr(lossy_ctx* ctx, float lr) {
   return LOSSY_OK;
 }
 
-int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat, uint8_t* count,
-                    uint64_t* recv_bits, void* stream) {
-  if (!ctx) return LOSSY_EINVAL;
+static int aggregate_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* ghat,
+                          uint8_t* count, uint64_t* recv_bits, void* stream) {
   if (ctx->cfg.n == 0) return LOSSY_OK;
   if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
   if (!ghat || !aligned16(ghat)) return fail(ctx, LOSSY_EINVAL, "ghat: NULL or misaligned");
@@ -276,9 +275,30 @@ int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads, flo
   fill_common(ctx, step, P);
   for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.grads[i] = grads[i];
   P.ghat = ghat;
+  P.ghat_prev = ghat_prev;
   P.count = count;
   P.recv_bits = recv_bits;
   return dispatch<AGG>(ctx, P, (cudaStream_t)stream, nullptr);
+}
+
+int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat, uint8_t* count,
+                    uint64_t* recv_bits, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  return aggregate_impl(ctx, step, grads, nullptr, ghat, count, recv_bits, stream);
+}
+
+static int check_alg1(lossy_ctx* ctx, const float* ghat_prev) {
+  if (ctx->cfg.flags & LOSSY_SELF_LOSSLESS)
+    return fail(ctx, LOSSY_EINVAL, "LOSSY_SELF_LOSSLESS has no meaning in Algorithm 1 mode");
+  if (ctx->cfg.n && (!ghat_prev || !aligned16(ghat_prev))) return fail(ctx, LOSSY_EINVAL, "ghat_prev: NULL or misaligned");
+  return LOSSY_OK;
+}
+
+int lossy_aggregate_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* ghat,
+                         uint8_t* count, uint64_t* recv_bits, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (int rc = check_alg1(ctx, ghat_prev)) return rc;
+  return aggregate_impl(ctx, step, grads, ghat_prev, ghat, count, recv_bits, stream);
 }
 
 int lossy_step(lossy_ctx* ctx, uint64_t step, const float* ghat, const uint8_t* count, float* master, float* m,
@@ -335,10 +355,9 @@ int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas
   return finalize_drift(ctx, blocks, norms, sumsq, (cudaStream_t)stream);
 }
 
-int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* master, float* m, float* v,
-                     void* const* replicas, float* ghat, uint8_t* count, uint64_t* recv_bits, uint64_t* stale_bits,
-                     float* norms, double* sumsq, void* stream) {
-  if (!ctx) return LOSSY_EINVAL;
+static int fused_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* master,
+                      float* m, float* v, void* const* replicas, float* ghat, uint8_t* count, uint64_t* recv_bits,
+                      uint64_t* stale_bits, float* norms, double* sumsq, void* stream) {
   if (step == 0) return fail(ctx, LOSSY_EINVAL, "step is 1-based");
   if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
   if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
@@ -363,6 +382,7 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, fl
   P.m = m;
   P.v = v;
   P.ghat = ghat;
+  P.ghat_prev = ghat_prev;
   P.count = count;
   P.recv_bits = recv_bits;
   P.stale_bits = stale_bits;
@@ -384,6 +404,23 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, fl
     rows += blocks;
   }
   return drift ? finalize_drift(ctx, rows, norms, sumsq, s) : LOSSY_OK;
+}
+
+int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* master, float* m, float* v,
+                     void* const* replicas, float* ghat, uint8_t* count, uint64_t* recv_bits, uint64_t* stale_bits,
+                     float* norms, double* sumsq, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  return fused_impl(ctx, step, grads, nullptr, master, m, v, replicas, ghat, count, recv_bits, stale_bits, norms, sumsq,
+                    stream);
+}
+
+int lossy_fused_step_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* master,
+                          float* m, float* v, void* const* replicas, float* ghat, uint8_t* count,
+                          uint64_t* recv_bits, uint64_t* stale_bits, float* norms, double* sumsq, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (int rc = check_alg1(ctx, ghat_prev)) return rc;
+  return fused_impl(ctx, step, grads, ghat_prev, master, m, v, replicas, ghat, count, recv_bits, stale_bits, norms,
+                    sumsq, stream);
 }
 
 int lossy_device_status(lossy_ctx* ctx, void* stream) {

@@ -33,6 +33,7 @@ struct Params {
   float* m;
   float* v;
   float* ghat;            // AGG: optional output; STEP without AGG: input
+  float* ghat_prev;       // non-NULL: Algorithm 1's gradient half (last surviving aggregate, in/out)
   uint8_t* count;         // optional output (AGG)
   uint64_t* recv_bits;    // optional output (AGG)
   uint64_t* stale_bits;   // optional output (BCAST)

@@ -36,10 +36,14 @@ __device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32
   const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k);
   const uint32_t i0 = lane, i1 = lane + 32;
   if constexpr (PH & AGG) {
-    bool s0 = i0 < W && (pair_hash(pkey, i0, j) >= P.Tg || ((P.flags & 1u) && i0 == j));
+    // Algorithm 1's gradient half: the reduce is reliable and ONE draw (the owner's own link of the
+    // hash) keeps or drops the packet's whole aggregate; otherwise one draw per contributing worker.
+    const bool alg1 = P.ghat_prev != nullptr;
+    const uint32_t src0 = alg1 ? j : i0, src1 = alg1 ? j : i1;
+    bool s0 = i0 < W && (pair_hash(pkey, src0, j) >= P.Tg || (!alg1 && (P.flags & 1u) && i0 == j));
     uint32_t lo = __ballot_sync(0xFFFFFFFFu, s0), hi = 0;
     if (W > 32) {
-      bool s1 = i1 < W && (pair_hash(pkey, i1, j) >= P.Tg || ((P.flags & 1u) && i1 == j));
+      bool s1 = i1 < W && (pair_hash(pkey, src1, j) >= P.Tg || (!alg1 && (P.flags & 1u) && i1 == j));
       hi = __ballot_sync(0xFFFFFFFFu, s1);
     }
     recv = ((uint64_t)hi << 32) | lo;
@@ -164,6 +168,15 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
         const float fc = (float)cnt;
 #pragma unroll
         for (int x = 0; x < 8; ++x) g[x] = __fdiv_rn(g[x], fc);
+      }
+      if (P.ghat_prev) {
+        // Algorithm 1: a dropped packet falls back to the saved aggregate, a surviving one is saved
+        if (cnt == 0) {
+          const Vec8<F32> pv = load8_any<F32>(P.ghat_prev, e, nvalid);
+          widen<F32>(pv, g);
+        } else {
+          store8<F32>(P.ghat_prev, e, narrow<F32>(g), nvalid);
+        }
       }
       if (P.ghat) {
         Vec8<F32> o = narrow<F32>(g);

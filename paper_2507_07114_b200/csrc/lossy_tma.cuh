@@ -242,6 +242,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if ((stale >> i) & 1ull)
             bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
       }
+      if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
       for (uint32_t g = 0; g < G.groups; ++g, ++it) {
         const uint32_t s = it % S, par = (it / S) & 1u;
         if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
@@ -352,6 +353,18 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             const float fc = (float)cnt;
 #pragma unroll
             for (int x = 0; x < kEpl; ++x) acc[x] = __fdiv_rn(acc[x], fc);
+          }
+          if (P.ghat_prev) {
+            // Algorithm 1: a dropped packet falls back to the saved aggregate, a surviving one is saved
+            uint32_t pw[4];
+            if (cnt == 0) {
+              load_words_stream<kEpl>(P.ghat_prev + e0 + idx, pw);
+              unpack_lane<F32>(pw, acc);
+            } else {
+#pragma unroll
+              for (int x = 0; x < kEpl; ++x) pw[x] = __float_as_uint(acc[x]);
+              __stcs(reinterpret_cast<uint4*>(P.ghat_prev + e0 + idx), make_uint4(pw[0], pw[1], pw[2], pw[3]));
+            }
           }
           if (P.ghat) {
             uint32_t gw[4];

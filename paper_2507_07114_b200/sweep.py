@@ -1,6 +1,6 @@
 """Throughput and drift of the fused step over the benchmark configurations.
 
-    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,5] [--steps N]
+    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,5,alg1] [--steps N]
 
 Prints one line per point: algorithmic GB/s, fraction of the measured HBM copy peak, steps/s and the
 largest per-replica drift norm seen. Inputs are the seeded synthetic workloads; state stays in HBM.
@@ -27,13 +27,15 @@ def _peak():
         return 6650.0
 
 
-def algorithmic_bytes(w):
+def algorithmic_bytes(w, alg1=False):
     gb = 2 if w.grad_dtype == "bf16" else 4
     rb = 2 if w.replica_dtype == "bf16" else 4
-    return (1.0 - w.p) * w.W * w.n * gb + (24 if w.optimizer == "adam" else 8) * w.n + w.W * w.n * rb
+    b = (1.0 - w.p) * w.W * w.n * gb + (24 if w.optimizer == "adam" else 8) * w.n + w.W * w.n * rb
+    # Algorithm 1 mode: the saved aggregate is read on a drop and written on a keep: 4 bytes per element
+    return b + (4 * w.n if alg1 else 0)
 
 
-def run_point(w, steps, warmup=3, grad_sets=2):
+def run_point(w, steps, warmup=3, grad_sets=2, alg1=False):
     dev = torch.device("cuda")
     gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
     rdt = torch.bfloat16 if w.replica_dtype == "bf16" else torch.float32
@@ -47,26 +49,34 @@ def run_point(w, steps, warmup=3, grad_sets=2):
     reps = [master.to(rdt) for _ in range(w.W)]
     norms = torch.zeros(w.W, device=dev)
     worst = torch.zeros(w.W, device=dev)
+    prev = torch.zeros_like(master) if alg1 else None
+
+    def step(t):
+        if alg1:
+            L.lossy_fused_step_alg1(ctx, t, sets[t % grad_sets], prev, master, m, v, reps, norms=norms)
+        else:
+            L.lossy_fused_step(ctx, t, sets[t % grad_sets], master, m, v, reps, norms=norms)
+
     sets = [[workload.grad_slab(w, s, i, 0, w.n, dev) for i in range(w.W)] for s in range(1, grad_sets + 1)]
     t = 0
     for _ in range(warmup):
         t += 1
-        L.lossy_fused_step(ctx, t, sets[t % grad_sets], master, m, v, reps, norms=norms)
+        step(t)
         torch.maximum(worst, norms, out=worst)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
         t += 1
-        L.lossy_fused_step(ctx, t, sets[t % grad_sets], master, m, v, reps, norms=norms)
+        step(t)
         torch.maximum(worst, norms, out=worst)
     e1.record()
     torch.cuda.synchronize()
     L.lossy_device_status(ctx)
     ms = e0.elapsed_time(e1) / steps
     L.lossy_destroy(ctx)
-    gbs = algorithmic_bytes(w) / (ms * 1e-3) / 1e9
-    return {"workload": w.name, "W": w.W, "P": w.packet_elems, "p": w.p, "ms_per_step": ms, "GBps": gbs,
+    gbs = algorithmic_bytes(w, alg1) / (ms * 1e-3) / 1e9
+    return {"workload": w.name + ("[alg1]" if alg1 else ""), "W": w.W, "P": w.packet_elems, "p": w.p, "ms_per_step": ms, "GBps": gbs,
             "frac_of_measured_peak": gbs / _peak(), "steps_per_s": 1e3 / ms, "max_drift_norm": float(worst.max())}
 
 
@@ -92,6 +102,13 @@ def main():
     for w in points:
         r = run_point(w, args.steps or w.steps, grad_sets=1 if w.W >= 64 else 2)
         print(json.dumps(r), flush=True)
+    if "alg1" in want:
+        # Algorithm 1 mode on the config-2 bucket: packet-granular and shard-granular (P = n / W) drops
+        base = cfg["cfg2_w8_layer_adam"]
+        for P in (2048, workload.LAYER_ELEMS // 8):
+            for p in (0.1, 0.3):
+                w = workload.scaled(base, base.n, packet_elems=P, p=p, name=f"cfg2_w8_P{P}_p{p}")
+                print(json.dumps(run_point(w, args.steps or 30, alg1=True)), flush=True)
 
 
 if __name__ == "__main__":

@@ -61,8 +61,9 @@ def assert_same(got, want, what):
 class GpuRun:
     """State of one simulated run on the GPU, advanced through the C ABI."""
 
-    def __init__(self, w: workload.Workload, *, flags=0, p_grad=None, p_param=None, theta0=None, device="cuda"):
-        self.w, self.dev = w, device
+    def __init__(self, w: workload.Workload, *, flags=0, p_grad=None, p_param=None, theta0=None, device="cuda",
+                 alg1=False):
+        self.w, self.dev, self.alg1 = w, device, alg1
         self.ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems,
                                 p_grad=w.p if p_grad is None else p_grad,
                                 p_param=w.p if p_param is None else p_param, seed=w.seed,
@@ -76,6 +77,7 @@ class GpuRun:
         self.v = torch.zeros(n, dtype=torch.float32, device=device)
         self.replicas = [self.master.to(tdtype(w.replica_dtype)).clone() for _ in range(W)]
         self.ghat = torch.zeros(n, dtype=torch.float32, device=device)
+        self.ghat_prev = torch.zeros(n, dtype=torch.float32, device=device) if alg1 else None
         self.count = torch.zeros(K, dtype=torch.uint8, device=device)
         self.recv = torch.zeros(K, dtype=torch.int64, device=device)
         self.stale = torch.zeros(K, dtype=torch.int64, device=device)
@@ -96,7 +98,11 @@ class GpuRun:
     def step_fused(self, t, grads, outputs=True):
         adam = self.w.optimizer == "adam"
         self.sumsq.zero_()
-        if outputs:
+        if self.alg1:
+            L.lossy_fused_step_alg1(self.ctx, t, grads, self.ghat_prev, self.master, self.m if adam else None,
+                                    self.v if adam else None, self.replicas, self.ghat, self.count, self.recv,
+                                    self.stale, self.norms, self.sumsq)
+        elif outputs:
             L.lossy_fused_step(self.ctx, t, grads, self.master, self.m if adam else None, self.v if adam else None,
                                self.replicas, self.ghat, self.count, self.recv, self.stale, self.norms, self.sumsq)
         else:
@@ -106,7 +112,10 @@ class GpuRun:
     def step_unfused(self, t, grads):
         adam = self.w.optimizer == "adam"
         self.sumsq.zero_()
-        L.lossy_aggregate(self.ctx, t, grads, self.ghat, self.count, self.recv)
+        if self.alg1:
+            L.lossy_aggregate_alg1(self.ctx, t, grads, self.ghat_prev, self.ghat, self.count, self.recv)
+        else:
+            L.lossy_aggregate(self.ctx, t, grads, self.ghat, self.count, self.recv)
         L.lossy_step(self.ctx, t, self.ghat, self.count, self.master, self.m if adam else None,
                      self.v if adam else None)
         L.lossy_broadcast(self.ctx, t, self.master, self.replicas, self.stale)
@@ -120,14 +129,14 @@ class GpuRun:
 
 
 def make_oracle(w: workload.Workload, *, flags=0, p_grad=None, p_param=None, theta0=None, k0=0, n_slab=None,
-                e0=0):
+                e0=0, alg1=False):
     n_slab = w.n - e0 if n_slab is None else n_slab
     th = workload.theta0_slab(w, e0, e0 + n_slab) if theta0 is None else theta0
     return O.Oracle(W=w.W, n=w.n, packet_elems=w.packet_elems, p_grad=w.p if p_grad is None else p_grad,
                     p_param=w.p if p_param is None else p_param, seed=w.seed, grad_dtype=odtype(w.grad_dtype),
                     replica_dtype=odtype(w.replica_dtype), optimizer=O.ADAM if w.optimizer == "adam" else O.SGD,
                     theta0=to_np(th), lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, flags=flags,
-                    packet_base=w.packet_base, k0=k0, n_slab=n_slab)
+                    packet_base=w.packet_base, k0=k0, n_slab=n_slab, alg1=alg1)
 
 
 def compare_state(gpu: GpuRun, orc, what, e0=0, e1=None):
@@ -150,10 +159,11 @@ def compare_outputs(out, ref, what, with_ghat=True):
     assert_rel(out["sumsq"], ref["sumsq"], f"{what} sumsq", tol=2 * REL_TOL)
 
 
-def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None, p_param=None, exact=True):
+def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None, p_param=None, exact=True,
+               alg1=False):
     """Element-by-element parity of a whole (small) run. Returns the GpuRun for further checks."""
-    gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param)
-    orc = make_oracle(w, flags=flags & 3, p_grad=p_grad, p_param=p_param)   # bit 4 only picks the kernel
+    gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param, alg1=alg1)
+    orc = make_oracle(w, flags=flags & 3, p_grad=p_grad, p_param=p_param, alg1=alg1)   # bit 4 only picks the kernel
     for t in range(1, steps + 1):
         gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]
         gd = [g.cuda() for g in gs]
@@ -161,6 +171,8 @@ def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None,
         ref = orc.step(t, [to_np(g) for g in gs])
         compare_outputs(gpu.outputs(), ref, f"{w.name} step {t}")
         compare_state(gpu, orc, f"{w.name} step {t}")
+        if alg1:
+            assert_same(to_np(gpu.ghat_prev), orc.ghat_prev, f"{w.name} step {t} ghat_prev")
     L.lossy_device_status(gpu.ctx)      # raises if a bounded wait inside a kernel gave up
     if exact:
         # fixed order + separately rounded operations on both sides: the state is in fact bit-identical
