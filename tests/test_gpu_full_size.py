@@ -81,3 +81,35 @@ def test_config5_point_full_size_small_packets_register_path():
     # P=256 takes the register-path kernel at full size
     w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.3)
     _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
+
+
+def test_drift_is_order_one_and_matches_the_stationary_constant_at_scale():
+    """Bounded Model Drift at scale, as a property that holds at any size: with SGD and gradients
+    redrawn i.i.d. every step, a replica's squared distance from the owners' values settles at
+    (elements it does not own) * p/(1-p) * sigma^2, sigma^2 = lr^2 sigma_g^2 E[1/c; c>0] — the
+    replica-vs-owner form of the theorem's constant — and does not grow with t."""
+    from math import comb
+
+    W, p, lr, sg = 8, 0.3, 1e-2, 1e-3
+    n = 2048 * 24000
+    w = workload.Workload("drift_at_scale", W, n, 2048, p, "sgd", lr, "bf16", "f32", 60, grad_sigma=sg, seed=4)
+    gpu = GpuRun(w)
+    hist = []
+    for t in range(1, 61):
+        gd = [workload.grad_slab(w, t, i, 0, n, "cuda") for i in range(W)]
+        gpu.step_fused(t, gd, outputs=False)
+        hist.append(gpu.norms.double().cpu().numpy() ** 2)
+        del gd
+    L.lossy_device_status(gpu.ctx)
+    inv_c = sum(comb(W, c) * (1 - p) ** c * p ** (W - c) / c for c in range(1, W + 1))
+    sigma2 = (lr * sg) ** 2 * inv_c
+    K = w.K
+    pps = (K + W - 1) // W
+    own = np.array([min(K, (i + 1) * pps) - min(K, i * pps) for i in range(W)]) * 2048
+    want = (n - own) * p / (1 - p) * sigma2
+    late = np.mean(hist[30:], axis=0)
+    assert np.all(np.abs(late / want - 1) < 0.03), (late / want)
+    first, second = np.mean(hist[20:40], axis=0), np.mean(hist[40:], axis=0)
+    assert np.all(np.abs(second / first - 1) < 0.03)                 # O(1): no growth with t
+    paper = (n - own) * 2 * p / (1 + p) * sigma2                     # the printed pairwise constant, for scale
+    assert np.all(late < 2.0 * paper)
