@@ -265,3 +265,26 @@ int NAME(drift_sumsq)(const oracle_config* c, uint64_t n_slab, const REAL* maste
   }
   return 0;
 }
+
+/*
+ * Closed-loop stand-in for "(1) Local gradient computation" of Section 3: worker i evaluates the
+ * gradient of a diagonal quadratic, L(theta) = 1/2 sum_e a[e] (theta[e] - x*[e])^2, at ITS OWN
+ * (possibly stale) replica and adds its mini-batch noise:
+ *     g_i[e] = cast( a[e] * (replica_i[e] - x*[e]) + noise_i[e] )
+ * sub, mul, add each rounded on its own; cast = identity (fp32 gradients) or RNE to bf16.
+ */
+int NAME(closed_loop_grads)(const oracle_config* c, uint64_t n_slab, const float* curv, const float* target,
+                            const void* const* noise, const void* const* replicas, void* const* grads_out) {
+  if (!c || !curv || !target || !noise || !replicas || !grads_out) return 1;
+  for (uint32_t i = 0; i < c->W; ++i)
+    for (uint64_t e = 0; e < n_slab; ++e) {
+      REAL rep = c->replica_dtype == DT_BF16 ? (REAL)bf16_to_f32(((const uint16_t*)replicas[i])[e])
+                                             : (REAL)((const float*)replicas[i])[e];
+      REAL d = rep - (REAL)target[e];
+      REAL q = (REAL)curv[e] * d;
+      REAL r = q + load_grad(noise[i], c->grad_dtype, e);
+      if (c->grad_dtype == DT_BF16) ((uint16_t*)grads_out[i])[e] = NAME(f32_to_bf16)((float)r);
+      else ((float*)grads_out[i])[e] = (float)r;
+    }
+  return 0;
+}

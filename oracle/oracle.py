@@ -82,6 +82,9 @@ def _lib(f64: bool):
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
         ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
+        cl = getattr(lib, pre + "closed_loop_grads")
+        cl.restype = C.c_int
+        cl.argtypes = [C.POINTER(OracleConfig), C.c_uint64] + [C.c_void_p] * 5
         _libs[key] = (lib, pre)
     return _libs[key]
 
@@ -184,6 +187,21 @@ class Oracle:
             raise ValueError("oracle_step rejected its arguments")
         return {"ghat": ghat, "count": count, "recv_bits": recv, "stale_bits": stale,
                 "sumsq": sumsq, "norms": np.sqrt(sumsq)}
+
+    def closed_loop_grads(self, curv, target, noise):
+        """Gradients of the diagonal quadratic evaluated at each worker's own replica, plus its noise."""
+        gd = np.uint16 if self.grad_dtype == BF16 else np.float32
+        curv = np.ascontiguousarray(curv, dtype=np.float32)
+        target = np.ascontiguousarray(target, dtype=np.float32)
+        noise = [np.ascontiguousarray(x, dtype=gd) for x in noise]
+        out = [np.zeros(self.n_slab, gd) for _ in range(self.W)]
+        nt, rt, ot = _ptr_table(noise), _ptr_table(self.replicas), _ptr_table(out)
+        rc = getattr(self.lib, self.pre + "closed_loop_grads")(
+            C.byref(self.cfg), self.n_slab, _ptr(curv), _ptr(target), C.cast(nt, C.c_void_p),
+            C.cast(rt, C.c_void_p), C.cast(ot, C.c_void_p))
+        if rc != 0:
+            raise ValueError("oracle_closed_loop_grads rejected its arguments")
+        return out
 
     def drift_sumsq(self):
         """Standalone drift: sum_e (replica_i[e] - cast(master[e]))^2 per replica, in double."""
