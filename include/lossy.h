@@ -246,6 +246,25 @@ int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host
                           void* stream);
 
 /*
+ * lossy_closed_loop_grads — a stand-in for Section 3 step (1), "local gradient
+ * computation", that restores the feedback the paper describes there: worker i
+ * computes its gradient at ITS OWN, possibly stale, replica. The objective is a
+ * diagonal quadratic, L(theta) = 1/2 sum_e a[e] (theta[e] - x*[e])^2, so
+ *     g_i[e] = cast( a[e] * (float(replica_i[e]) - x*[e]) + float(noise_i[e]) ),
+ * subtraction, multiplication and addition each rounded to fp32 on their own,
+ * cast = identity or RNE to bf16 (cfg.grad_dtype). Call it before
+ * lossy_fused_step to run the method in closed loop on synthetic data.
+ *   curv, target  [n] fp32 device (a and x*)
+ *   noise         host array of W device pointers, each [n] of cfg.grad_dtype
+ *                 (the mini-batch noise of worker i, drawn by the caller)
+ *   replicas      host array of W device pointers, each [n] of cfg.replica_dtype
+ *   grads_out     host array of W device pointers, each [n] of cfg.grad_dtype, written
+ */
+int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* target,
+                            const void* const* noise, const void* const* replicas,
+                            void* const* grads_out, void* stream);
+
+/*
  * lossy_device_status — synchronise `stream` and report whether any kernel of
  * this context gave up a bounded wait (the bulk-copy pipeline bounds every wait
  * on its barriers instead of spinning forever). LOSSY_OK, or LOSSY_EDEVICE if

@@ -22,7 +22,7 @@ LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_aggregate", "lossy_step", "lossy_broadcast",
     "drift_norms", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
-    "lossy_mask_grid", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
+    "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
 
 
@@ -86,6 +86,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_hash_u32.argtypes = [u64, u64, u32, u32, u64]
     lib.lossy_mask_grid.restype = C.c_int
     lib.lossy_mask_grid.argtypes = [vp, u64, vp, vp, vp, u64, C.c_int, vp, vp]
+    lib.lossy_closed_loop_grads.restype = C.c_int
+    lib.lossy_closed_loop_grads.argtypes = [vp] * 7
     lib.lossy_device_status.restype = C.c_int
     lib.lossy_device_status.argtypes = [vp, vp]
     lib.lossy_last_error.restype = C.c_char_p
@@ -215,6 +217,11 @@ def lossy_hash_u32(seed, step, src, dst, packet) -> int:
 def lossy_mask_grid(ctx, step, src, dst, packet, out, is_param=False):
     _check(ctx, load_library().lossy_mask_grid(ctx, step, _p(src), _p(dst), _p(packet), src.numel(), int(is_param),
                                                _p(out), _stream()))
+
+
+def lossy_closed_loop_grads(ctx, curv, target, noise, replicas, grads_out):
+    _check(ctx, load_library().lossy_closed_loop_grads(ctx, _p(curv), _p(target), _table(noise), _table(replicas),
+                                                       _table(grads_out), _stream()))
 
 
 def lossy_device_status(ctx):

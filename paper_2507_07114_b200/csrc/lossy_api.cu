@@ -423,6 +423,41 @@ int lossy_fused_step_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grad
                     sumsq, stream);
 }
 
+int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* target, const void* const* noise,
+                            const void* const* replicas, void* const* grads_out, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  if (!curv || !target || !aligned16(curv) || !aligned16(target)) return fail(ctx, LOSSY_EINVAL, "curv/target: NULL or misaligned");
+  if (int rc = check_table(ctx, noise, "noise: NULL or misaligned pointer")) return rc;
+  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (int rc = check_table(ctx, grads_out, "grads_out: NULL or misaligned pointer")) return rc;
+  ClosedLoopArgs A;
+  memset(&A, 0, sizeof A);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) {
+    A.noise[i] = noise[i];
+    A.replicas[i] = replicas[i];
+    A.grads[i] = grads_out[i];
+  }
+  A.curv = curv;
+  A.target = target;
+  A.n = ctx->cfg.n;
+  A.W = ctx->cfg.W;
+  const uint64_t nvec = (A.n + 7) / 8;
+  uint64_t blocks = (nvec + 255) / 256;
+  const uint64_t cap = (uint64_t)ctx->num_sms * 8;
+  if (blocks > cap) blocks = cap;
+  const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16, rb = ctx->cfg.replica_dtype == LOSSY_BF16;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (gb && rb) closed_loop_grads_kernel<BF16, BF16><<<(uint32_t)blocks, 256, 0, s>>>(A);
+  else if (gb) closed_loop_grads_kernel<BF16, F32><<<(uint32_t)blocks, 256, 0, s>>>(A);
+  else if (rb) closed_loop_grads_kernel<F32, BF16><<<(uint32_t)blocks, 256, 0, s>>>(A);
+  else closed_loop_grads_kernel<F32, F32><<<(uint32_t)blocks, 256, 0, s>>>(A);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "closed-loop gradient launch", e);
+  ctx->launches++;
+  return LOSSY_OK;
+}
+
 int lossy_device_status(lossy_ctx* ctx, void* stream) {
   if (!ctx) return LOSSY_EINVAL;
   uint32_t word = 0;

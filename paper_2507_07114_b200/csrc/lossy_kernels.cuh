@@ -287,6 +287,51 @@ static __global__ void drift_finalize_kernel(const double* __restrict__ partials
   }
 }
 
+// Closed-loop stand-in for the local gradient computation (Section 3 step (1)): worker i's gradient of
+// 1/2 sum a (theta - x*)^2 at ITS OWN replica plus its noise, g_i = cast(a * (replica_i - x*) + noise_i),
+// each operation rounded on its own. One lane per 8 elements, workers four at a time.
+struct ClosedLoopArgs {
+  const void* noise[kMaxW];
+  const void* replicas[kMaxW];
+  void* grads[kMaxW];
+  const float* curv;
+  const float* target;
+  uint64_t n;
+  uint32_t W;
+};
+
+template <class GT, class RT>
+static __global__ void __launch_bounds__(256) closed_loop_grads_kernel(const __grid_constant__ ClosedLoopArgs A) {
+  const uint64_t nvec = (A.n + 7) / 8;
+  for (uint64_t vi = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t e = vi * 8;
+    const int nvalid = A.n - e >= 8 ? 8 : (int)(A.n - e);
+    float a[8], xs[8];
+    widen<F32>(load8_any<F32>(A.curv, e, nvalid), a);
+    widen<F32>(load8_any<F32>(A.target, e, nvalid), xs);
+    for (uint32_t i0 = 0; i0 < A.W; i0 += 4) {
+      Vec8<RT> rep[4];
+      Vec8<GT> nz[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (i0 + u < A.W) {
+          rep[u] = load8_any<RT>(A.replicas[i0 + u], e, nvalid);
+          nz[u] = load8_any<GT>(A.noise[i0 + u], e, nvalid);
+        }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (i0 + u < A.W) {
+          float r[8], z[8], g[8];
+          widen<RT>(rep[u], r);
+          widen<GT>(nz[u], z);
+#pragma unroll
+          for (int x = 0; x < 8; ++x) g[x] = __fadd_rn(__fmul_rn(a[x], __fsub_rn(r[x], xs[x])), z[x]);
+          store8<GT>(A.grads[i0 + u], e, narrow<GT>(g), nvalid);
+        }
+    }
+  }
+}
+
 // Delivery indicators on a dense grid of tuples (host/device agreement check).
 static __global__ void mask_grid_kernel(uint64_t seed, uint64_t step, const uint32_t* src, const uint32_t* dst,
                                  const uint64_t* packet, uint64_t count, uint32_t T, uint8_t* out) {

@@ -1,0 +1,49 @@
+"""Closed loop on the GPU (gradient stand-in kernel + fused step) against the oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2507_07114_b200 as L
+import workload
+from parity_util import GpuRun, assert_same, compare_state, make_oracle, to_np
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    ("sgd_f32", 4, 1024 * 19 + 5, 1024, 0.3, "sgd", 0.1, "f32", "f32"),
+    ("adam_bf16", 8, 2048 * 11 + 24, 2048, 0.2, "adam", 3e-3, "bf16", "bf16"),
+    ("w33_mixed", 33, 256 * 40, 256, 0.1, "sgd", 0.05, "bf16", "f32"),
+    ("f32_grads_bf16_replicas", 5, 1024 * 7, 1024, 0.4, "adam", 1e-3, "f32", "bf16"),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_closed_loop_matches_the_oracle(case):
+    name, W, n, P, p, opt, lr, gd, rd = case
+    w = workload.Workload("cl_" + name, W, n, P, p, opt, lr, gd, rd, 8, seed=5)
+    gpu, orc = GpuRun(w), make_oracle(w)
+    curv = 0.5 + workload.normal_f32(5, 4000, 0, 0, n, 1.0).abs() % 1.0
+    target = workload.normal_f32(5, 4001, 0, 0, n, 1.0)
+    gdt = torch.bfloat16 if gd == "bf16" else torch.float32
+    grads = [torch.empty(n, dtype=gdt, device="cuda") for _ in range(W)]
+    curv_d, target_d = curv.cuda(), target.cuda()
+    for t in range(1, 9):
+        noise = [workload.normal_f32(5, 5000 + i, t, 0, n, 1.0).to(gdt) for i in range(W)]
+        L.lossy_closed_loop_grads(gpu.ctx, curv_d, target_d, [x.cuda() for x in noise], gpu.replicas, grads)
+        ref_g = orc.closed_loop_grads(curv.numpy(), target.numpy(), [to_np(x) for x in noise])
+        for i in range(W):
+            assert_same(to_np(grads[i]), ref_g[i], f"{name} step {t} gradient of worker {i}")
+        gpu.step_fused(t, grads)
+        orc.step(t, ref_g)
+        compare_state(gpu, orc, f"{name} step {t}")
+    assert_same(to_np(gpu.master), orc.master, f"{name} master bits")
+    L.lossy_device_status(gpu.ctx)
+
+
+def test_objective_degrades_gently_with_the_drop_rate():
+    from paper_2507_07114_b200.closed_loop import run
+
+    vals = [run(p, W=8, n=2048 * 512, P=2048, steps=120, optimizer="sgd", lr=0.1, gdt=torch.float32,
+                rdt=torch.float32)[0] for p in (0.0, 0.1, 0.3)]
+    assert vals[0] < vals[1] < vals[2]
+    assert vals[1] / vals[0] < 1.35 and vals[2] / vals[0] < 3.0
