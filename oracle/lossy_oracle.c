@@ -124,6 +124,13 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
  *                   Algorithm 1's gradient half — the reduce over all W workers is reliable,
  *                   then ONE draw per packet decides whether the owner keeps the fresh aggregate
  *                   (and saves it as "prev") or falls back to the saved previous aggregate
+ *   burst           NULL: independent Bernoulli drops (the paper's model). Non-NULL: double[2] =
+ *                   {P(good->bad), P(bad->good)} of a two-state (Gilbert-Elliott) chain per link
+ *                   and packet, the bursty loss the paper's Limitations leave open: with u the same
+ *                   hash value, bad_t = bad_{t-1} ? (u >= T_leave) : (u < T_enter), T = floor(p 2^32);
+ *                   a transmission is lost iff its link is bad at step t. p_grad / p_param are unused.
+ *   burst_in/out    [2][packets] uint64 (row 0 gradient links, row 1 broadcast links; bit i = link of
+ *                   worker i is bad): state after step t-1 (read) and after step t (written)
  *   recv_force      optional [packets] uint64: use these delivery bits (bit i = s_i)
  *                   instead of the hash — the hook the exhaustive-pattern test uses
  *                   (Algorithm 1 mode: bit 0 = the packet's aggregate survives)
@@ -136,7 +143,8 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
  */
 int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_slab,
                const void* const* grads, REAL* master, REAL* m, REAL* v, void* const* replicas,
-               REAL* ghat_prev, const uint64_t* recv_force, const uint64_t* stale_force,
+               REAL* ghat_prev, const double* burst, const uint64_t* burst_in, uint64_t* burst_out,
+               const uint64_t* recv_force, const uint64_t* stale_force,
                REAL* ghat, uint8_t* count, uint64_t* recv_bits, uint64_t* stale_bits,
                uint32_t* const* age, double* sumsq) {
   if (!c || c->W == 0 || c->W > 64 || c->packet_elems == 0) return 1;
@@ -147,6 +155,14 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
   const uint64_t slab_start = k0 * P;
   if (slab_start + n_slab > c->n) return 1;
   const uint64_t packets = (n_slab + P - 1) / P;
+  uint32_t Tenter = 0, Tleave = 0;
+  if (burst) {
+    if (!burst_in || !burst_out) return 1;
+    if (!(burst[0] >= 0.0 && burst[0] < 1.0) || !(burst[1] > 0.0 && burst[1] <= 1.0)) return 1;
+    Tenter = NAME(threshold)(burst[0]);
+    /* P(bad->good) = 1 means "always leave": the compare u >= T can then never fail */
+    Tleave = burst[1] >= 1.0 ? 0u : NAME(threshold)(1.0 - burst[1]);
+  }
 
   /* Adam's scalars: (1-beta) in fp32, bias corrections in double then rounded once. */
   const REAL lr = (REAL)c->lr, b1 = (REAL)c->beta1, b2 = (REAL)c->beta2, eps = (REAL)c->eps;
@@ -163,15 +179,34 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
 
     /* (2) which workers' pieces reached the owner: s^(i,j) */
     uint64_t recv = 0;
+    uint64_t gbad = 0, pbad = 0;   /* link states after this step (bursty mode) */
     if (ghat_prev) {
       /* Algorithm 1: "reduce-scatter" is lossless, then Uniform(0,1) < p_grad drops the whole packet */
-      int keep = recv_force ? (int)(recv_force[kl] & 1ULL) : (NAME(hash_u32)(c->seed, step, j, j, kg) >= Tg);
+      int keep;
+      if (recv_force) keep = (int)(recv_force[kl] & 1ULL);
+      else if (burst) {
+        uint32_t u = NAME(hash_u32)(c->seed, step, j, j, kg);
+        int was_bad = (int)(burst_in[kl] & 1ULL);
+        int bad = was_bad ? (u < Tleave) : (u < Tenter);
+        gbad = (uint64_t)bad;
+        keep = !bad;
+      } else keep = NAME(hash_u32)(c->seed, step, j, j, kg) >= Tg;
       if (keep) recv = W == 64 ? ~0ULL : ((1ULL << W) - 1ULL);
     } else if (recv_force) recv = recv_force[kl];
     else
       for (uint32_t i = 0; i < W; ++i) {
-        int s = NAME(hash_u32)(c->seed, step, i, j, kg) >= Tg;
-        if ((c->flags & FLAG_SELF_LOSSLESS) && i == j) s = 1;
+        uint32_t u = NAME(hash_u32)(c->seed, step, i, j, kg);
+        int s;
+        if (burst) {
+          int was_bad = (int)((burst_in[kl] >> i) & 1ULL);
+          int bad = was_bad ? (u < Tleave) : (u < Tenter);   /* stays bad unless u >= T_leave */
+          if ((c->flags & FLAG_SELF_LOSSLESS) && i == j) bad = 0;
+          if (bad) gbad |= 1ULL << i;
+          s = !bad;
+        } else {
+          s = u >= Tg;
+          if ((c->flags & FLAG_SELF_LOSSLESS) && i == j) s = 1;
+        }
         if (s) recv |= 1ULL << i;
       }
     uint32_t cnt = 0;
@@ -182,9 +217,18 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
     /* (4) which replicas take the broadcast of this packet: r^(j,i); the owner always has it */
     uint64_t stale = 0;
     if (stale_force) stale = stale_force[kl] & ~(1ULL << j);
-    else
+    else if (burst) {
+      for (uint32_t i = 0; i < W; ++i) {
+        if (i == j) continue;
+        uint32_t u = NAME(hash_u32)(c->seed, step, j, i, kg);
+        int was_bad = (int)((burst_in[packets + kl] >> i) & 1ULL);
+        int bad = was_bad ? (u < Tleave) : (u < Tenter);
+        if (bad) { pbad |= 1ULL << i; stale |= 1ULL << i; }
+      }
+    } else
       for (uint32_t i = 0; i < W; ++i)
         if (i != j && NAME(hash_u32)(c->seed, step, j, i, kg) < Tp) stale |= 1ULL << i;
+    if (burst) { burst_out[kl] = gbad; burst_out[packets + kl] = pbad; }
     if (stale_bits) stale_bits[kl] = stale;
 
     for (uint64_t e = e0; e < e1; ++e) {

@@ -78,7 +78,7 @@ def _lib(f64: bool):
         o.argtypes = [C.POINTER(OracleConfig), C.c_uint64]
         s = getattr(lib, pre + "step")
         s.restype = C.c_int
-        s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 14
+        s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 17
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
         ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -134,7 +134,7 @@ class Oracle:
 
     def __init__(self, *, W, n, packet_elems, p_grad, p_param, seed, grad_dtype, replica_dtype,
                  optimizer, theta0, lr, beta1=0.9, beta2=0.95, eps=1e-8, flags=0, packet_base=0,
-                 k0=0, n_slab=None, f64=False, track_age=False, alg1=False):
+                 k0=0, n_slab=None, f64=False, track_age=False, alg1=False, burst=None):
         self.cfg = OracleConfig(W, packet_elems, n, packet_base, p_grad, p_param, seed, grad_dtype,
                                 replica_dtype, optimizer, flags, lr, beta1, beta2, eps)
         self.W, self.P, self.n, self.k0 = W, packet_elems, n, k0
@@ -153,6 +153,9 @@ class Oracle:
         self.age = [np.zeros(self.packets, np.uint32) for _ in range(W)] if track_age else None
         # Algorithm 1's gradient half keeps the last surviving aggregate per element ("g_prev"), zero at start
         self.ghat_prev = np.zeros(self.n_slab, self.real) if alg1 else None
+        # bursty loss: (P(good->bad), P(bad->good)) and the link states [2][packets], all good at start
+        self.burst = None if burst is None else np.array(burst, dtype=np.float64)
+        self.burst_state = np.zeros((2, self.packets), np.uint64) if burst is not None else None
         self.grad_dtype, self.replica_dtype = grad_dtype, replica_dtype
 
     def owner(self, k: int) -> int:
@@ -177,14 +180,17 @@ class Oracle:
             recv_force = np.ascontiguousarray(recv_force, dtype=np.uint64)
         if stale_force is not None:
             stale_force = np.ascontiguousarray(stale_force, dtype=np.uint64)
+        burst_out = np.zeros_like(self.burst_state) if self.burst is not None else None
         rc = getattr(self.lib, self.pre + "step")(
             C.byref(self.cfg), t, self.k0, self.n_slab, C.cast(gt, C.c_void_p), _ptr(self.master),
-            _ptr(self.m), _ptr(self.v), C.cast(rt, C.c_void_p), _ptr(self.ghat_prev), _ptr(recv_force),
-            _ptr(stale_force),
+            _ptr(self.m), _ptr(self.v), C.cast(rt, C.c_void_p), _ptr(self.ghat_prev), _ptr(self.burst),
+            _ptr(self.burst_state), _ptr(burst_out), _ptr(recv_force), _ptr(stale_force),
             _ptr(ghat), _ptr(count), _ptr(recv), _ptr(stale),
             C.cast(at, C.c_void_p) if at is not None else None, _ptr(sumsq))
         if rc != 0:
             raise ValueError("oracle_step rejected its arguments")
+        if self.burst is not None:
+            self.burst_state = burst_out
         return {"ghat": ghat, "count": count, "recv_bits": recv, "stale_bits": stale,
                 "sumsq": sumsq, "norms": np.sqrt(sumsq)}
 
