@@ -81,12 +81,30 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
 constexpr uint32_t kTmaSmemFixed = 128 + kMaxStages * sizeof(StageHdr);
 
-// L2 evict-first hints on the bulk copies (bit 0 loads, bit 1 stores). Measured on B200: +3-4 % at
-// W = 64 (eight worker groups per tile), nothing at W = 32, about -1 % at W <= 16.
-uint32_t tma_hints(uint32_t groups) { return groups > 4 ? 3u : 0u; }
+// Launch policy of the bulk-copy pipeline, from sweeps on B200 over W = 2..64, p = 0.05..0.3
+// (bandwidths in profiles/): which of the four builds runs and whether its bulk copies carry an
+// L2 evict-first hint (bit 0 loads, bit 1 stores).
+struct TmaPolicy {
+  bool wide;      // 16 compute warps, one CTA per SM, 2048-element tiles (else 8 warps, two CTAs, 1024)
+  int group;      // workers per pipeline stage: 4 or 8
+  uint32_t hints;
+};
+TmaPolicy tma_policy(const lossy_config& c) {
+  const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
+  TmaPolicy t;
+  // wide tiles win whenever a tile takes at most two 8-worker groups and the packet is a multiple of the tile
+  t.wide = c.W <= 16 && c.packet_elems % TmaShape<16>::kTile == 0;
+  // stages of 4 workers (finer-grained pipeline) win for few workers at low loss: +5 % at W = 8, p = 0.1,
+  // but -9 % at W = 8, p = 0.3; the crossover at W = 8 sits near p = 0.17
+  t.group = c.W <= 4 ? 4 : (c.W <= 8 && pm < 0.175 ? 4 : 8);
+  // hints: +3-4 % on the twin build at W = 64 or at high loss, neutral to -2 % elsewhere
+  t.hints = t.wide ? (pm >= 0.28 ? 3u : 0u) : ((c.W > 32 || pm >= 0.2) ? 3u : 0u);
+  return t;
+}
 
-template <int CW>
+template <int CW, int GS>
 bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
+  constexpr uint32_t kGroup = GS;
   constexpr uint32_t kTile = TmaShape<CW>::kTile;
   const lossy_config& c = ctx->cfg;
   if (c.packet_elems < kTile) return false;
@@ -107,13 +125,13 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   if (tiles >= (1ull << 31)) return false;
   G.num_tiles = (uint32_t)tiles;
   G.status = ctx->status;
-  G.hints = tma_hints(G.groups);
+  G.hints = tma_policy(c).hints;
   return true;
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK, int CW>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS>
 int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW>;
+  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS>;
   constexpr int kThreadsTma = TmaShape<CW>::kThreads;
   const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -133,33 +151,36 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   return LOSSY_OK;
 }
 
-template <bool DRIFTK, int CW>
+template <bool DRIFTK, int CW, int GS>
 int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
   const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
   const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
   const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
-  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
-  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
-  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
-  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW>(ctx, P, G, s, blocks);
+  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
+  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
 }
 
-// Pick the geometry: wide tiles when a tile takes at most two worker groups and the packet is a
-// multiple of the wide tile (measured 3-4 % faster there), else the twin-CTA build; false = no bulk-copy launch (register path takes everything).
+template <int CW, int GS>
+int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
+  TmaGeom G;
+  if (!tma_geometry<CW, GS>(ctx, G)) return LOSSY_OK;
+  *used = true;
+  return drift ? dispatch_tma<true, CW, GS>(ctx, P, G, s, blocks) : dispatch_tma<false, CW, GS>(ctx, P, G, s, blocks);
+}
+
+// Run the build the policy picks; *used stays false when no bulk-copy launch fits (packets shorter
+// than a tile, or no complete packet): the register path then takes everything.
 int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
   *used = false;
   if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
-  TmaGeom G;
-  const bool wide_ok = ctx->cfg.W <= 2u * kGroup && ctx->cfg.packet_elems % TmaShape<16>::kTile == 0;
-  if (wide_ok && tma_geometry<16>(ctx, G)) {
-    *used = true;
-    return drift ? dispatch_tma<true, 16>(ctx, P, G, s, blocks) : dispatch_tma<false, 16>(ctx, P, G, s, blocks);
+  const TmaPolicy t = tma_policy(ctx->cfg);
+  if (t.wide) {
+    int rc = t.group == 4 ? try_tma<16, 4>(ctx, P, drift, s, blocks, used) : try_tma<16, 8>(ctx, P, drift, s, blocks, used);
+    if (rc || *used) return rc;
   }
-  if (tma_geometry<8>(ctx, G)) {
-    *used = true;
-    return drift ? dispatch_tma<true, 8>(ctx, P, G, s, blocks) : dispatch_tma<false, 8>(ctx, P, G, s, blocks);
-  }
-  return LOSSY_OK;
+  return t.group == 4 ? try_tma<8, 4>(ctx, P, drift, s, blocks, used) : try_tma<8, 8>(ctx, P, drift, s, blocks, used);
 }
 
 template <int PH, class GT, class RT, int OPT>

@@ -2,7 +2,7 @@
 //
 // One CTA = CW compute warps + 1 producer warp + 1 store warp (see TmaShape for the two builds).
 // The bucket's full packets are cut into tiles of at most kTile contiguous elements inside one
-// packet (kTile = 128 * CW), so one set of delivery masks covers a tile. Per tile and per group of up to 8 workers
+// packet (kTile = 128 * CW), so one set of delivery masks covers a tile. Per tile and per group of up to GS (4 or 8) workers
 // the producer arms an mbarrier and issues 1-D bulk copies global -> shared memory for the
 // DELIVERED workers' pieces only (dropped packets are never read) and, with the last group, for
 // theta / m / v. Compute warps sum the pieces in ascending worker order from shared memory,
@@ -22,15 +22,16 @@ namespace lossy {
 
 constexpr int kEpl = 4;                                   // elements per compute lane
 // Two geometries are built: "wide" = 16 compute warps, one CTA per SM, tiles of 2048 elements
-// (best when a tile takes one or two worker groups, W <= 16); "twin" = 8 compute warps, two CTAs
-// per SM, tiles of 1024 elements (best when a tile takes many worker groups).
+// (best for W <= 16); "twin" = 8 compute warps, two CTAs per SM, tiles of 1024 elements (best when
+// a tile takes many worker groups). Each comes with pipeline stages of 4 or of 8 workers (GS).
 template <int CW> struct TmaShape {
   static constexpr int kConsumerWarps = CW;
   static constexpr int kTile = CW * 32 * kEpl;
   static constexpr int kThreads = (CW + 2) * 32;          // + producer warp + store warp
   static constexpr int kCtasPerSm = CW >= 16 ? 1 : 2;
 };
-constexpr int kGroup = 8;                                 // workers per pipeline stage
+constexpr int kStaleBatch = 4;                            // stale replica packets in flight per compute lane (8 measured slower)
+constexpr int kGroupMax = 8;                              // workers per pipeline stage: template GS = 4 or 8
 constexpr int kMaxStages = 4;
 constexpr uint32_t kMaxPolls = 1u << 22;
 
@@ -39,8 +40,8 @@ struct TmaGeom {
   uint32_t tiles_per_packet;
   uint32_t stages;
   uint32_t stage_bytes;       // per stage, 128-byte multiple
-  uint32_t groups;            // ceil(W / kGroup)
-  uint32_t grad_slots;        // min(W, kGroup)
+  uint32_t groups;            // ceil(W / GS)
+  uint32_t grad_slots;        // min(W, GS)
   uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores
   uint32_t* status;           // device status word (0 = fine)
 };
@@ -180,10 +181,11 @@ __device__ __forceinline__ void pack_bf16_lane(const float (&f)[kEpl], uint32_t 
   }
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK, int CW>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS>
 __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPerSm)
     lossy_fused_tma_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
   constexpr int kConsumerWarps = CW;
+  constexpr int kGroup = GS;                // workers whose pieces share one pipeline stage
   constexpr int kTile = TmaShape<CW>::kTile;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
@@ -247,7 +249,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint32_t s = it % S, par = (it / S) & 1u;
         if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
         const bool last = g + 1 == G.groups;
-        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & 0xFFu;
+        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
         unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
         if (lane == 0) {
           StageHdr& h = hdrs[s];
@@ -328,7 +330,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
 #pragma unroll
           for (int x = 0; x < kEpl; ++x) acc[x] = 0.0f;
         }
-        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & 0xFFu;
+        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
         if (active) {
 #pragma unroll
           for (int u = 0; u < kGroup; ++u)
@@ -422,12 +424,12 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         if constexpr (DRIFTK) {
           uint64_t sm = stale;
           while (sm) {
-            // up to four stale copies are fetched before the first is used
-            int ids[4];
-            float old[4][kEpl];
+            // up to kStaleBatch stale copies are fetched before the first is used
+            int ids[kStaleBatch];
+            float old[kStaleBatch][kEpl];
             int nb = 0;
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < kStaleBatch; ++b) {
               ids[b] = -1;
               if (sm) {
                 ids[b] = __ffsll((long long)sm) - 1;
@@ -445,7 +447,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               }
             }
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < kStaleBatch; ++b) {
               if (b < nb) {
                 float sq = 0.0f;
 #pragma unroll
