@@ -38,9 +38,9 @@ WORKLOAD = "cfg2_w8_layer_adam"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the fused kernel, from the ncu capture
-# summarised in profiles/fused_step_cfg2_w8_layer.md: 1774.2 MB on a 33,554,432-element cut of the
+# summarised in profiles/fused_step_cfg2_w8_layer.md: 1769.7 MB on a 33,554,432-element cut of the
 # workload, scaled by the elements processed (traffic is proportional to them).
-NCU_TRAFFIC_SMALL_CASE = (1774.2e6, 33554432)
+NCU_TRAFFIC_SMALL_CASE = (1769.7e6, 33554432)
 
 
 def algorithmic_bytes(w: workload.Workload, n: int | None = None) -> float:
