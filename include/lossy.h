@@ -98,6 +98,27 @@ void lossy_destroy(lossy_ctx* ctx);
 int lossy_set_lr(lossy_ctx* ctx, float lr);
 
 /*
+ * lossy_set_bursty — replace the independent Bernoulli drops by bursty loss, the
+ * correlated regime the paper's Limitations section leaves open (its analysis
+ * assumes i.i.d. drops): every link (src -> dst) of every packet is a two-state
+ * Gilbert-Elliott chain driven by the SAME hash value u as the independent draw,
+ *     bad_t = bad_{t-1} ? (u < floor((1 - p_leave_bad) 2^32)) : (u < floor(p_enter_bad 2^32)),
+ * and a transmission is lost iff its link is bad at step t (p_grad / p_param are
+ * then unused). Stationary loss rate p_enter/(p_enter + p_leave), mean burst length
+ * 1/p_leave; p_enter = p, p_leave = 1 - p has the statistics of independent loss.
+ *   state   device, caller-owned, 4*K uint64 = [2 buffers][row 0 gradient links,
+ *           row 1 broadcast links][K], bit i = the link of worker i is bad; zero it
+ *           before step 1 (all links good). Step t reads buffer (t-1)&1 and writes
+ *           buffer t&1, so steps must be issued in order 1, 2, 3, ... and the array
+ *           belongs in a checkpoint. NULL switches back to independent loss.
+ * In Algorithm 1 mode the gradient half uses one chain per packet (bit 0).
+ * lossy_mask / lossy_mask_grid keep evaluating the independent draw.
+ * Errors: LOSSY_EINVAL (probabilities outside 0 <= p_enter < 1, 0 < p_leave <= 1;
+ * misaligned state).
+ */
+int lossy_set_bursty(lossy_ctx* ctx, double p_enter_bad, double p_leave_bad, uint64_t* state);
+
+/*
  * lossy_aggregate — Section 3 step (2) and "Unbiased Gradient Aggregation":
  * for every packet k with owner j,
  *     s_i   = 1 iff hash(seed, step, src=i, dst=j, packet_base+k) >= T_grad

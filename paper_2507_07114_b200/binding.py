@@ -20,7 +20,7 @@ LOSSY_SGD, LOSSY_ADAM = 0, 1
 LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 
 EXPORTS = [
-    "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_aggregate", "lossy_step", "lossy_broadcast",
+    "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_aggregate", "lossy_step", "lossy_broadcast",
     "drift_norms", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
@@ -62,6 +62,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_destroy.argtypes = [vp]
     lib.lossy_set_lr.restype = C.c_int
     lib.lossy_set_lr.argtypes = [vp, C.c_float]
+    lib.lossy_set_bursty.restype = C.c_int
+    lib.lossy_set_bursty.argtypes = [vp, C.c_double, C.c_double, vp]
     lib.lossy_aggregate.restype = C.c_int
     lib.lossy_aggregate.argtypes = [vp, u64, vp, vp, vp, vp, vp]
     lib.lossy_step.restype = C.c_int
@@ -148,6 +150,11 @@ def lossy_destroy(ctx):
 
 def lossy_set_lr(ctx, lr):
     _check(ctx, load_library().lossy_set_lr(ctx, lr))
+
+
+def lossy_set_bursty(ctx, p_enter_bad, p_leave_bad, state):
+    """state: int64/uint64 device tensor of 4*K elements, zeroed before step 1; None = independent loss."""
+    _check(ctx, load_library().lossy_set_bursty(ctx, p_enter_bad, p_leave_bad, _p(state)))
 
 
 def lossy_aggregate(ctx, step, grads, ghat, count=None, recv_bits=None):

@@ -24,6 +24,8 @@ struct lossy_ctx {
   uint32_t max_blocks;   // capacity of `partials`
   double* partials;      // device, [max_blocks][kMaxW], followed by the status word
   uint32_t* status;      // device status word: 0 = fine, 1 = a bounded wait in a kernel gave up
+  uint64_t* burst_state; // bursty loss: caller-owned device array [2 buffers][2 rows][K], or NULL
+  uint32_t Tenter, Tstay;
   int smem_optin;        // largest dynamic shared memory a block may opt in to
   uint64_t launches;
   char err[256];
@@ -76,6 +78,15 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   P.ibc2 = (float)(1.0 / (1.0 - pow((double)c.beta2, (double)step)));
   P.eps = c.eps;
   P.partials = ctx->partials;
+  P.K = (uint32_t)ctx->K;
+  if (ctx->burst_state) {
+    // the states after step t-1 live in buffer (t-1)&1, those after step t go to buffer t&1
+    const size_t buf = 2 * (size_t)ctx->K;
+    P.burst_in = ctx->burst_state + ((step - 1) & 1u) * buf;
+    P.burst_out = ctx->burst_state + (step & 1u) * buf;
+    P.Tenter = ctx->Tenter;
+    P.Tstay = ctx->Tstay;
+  }
 }
 
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
@@ -279,6 +290,22 @@ void lossy_destroy(lossy_ctx* ctx) {
   if (!ctx) return;
   if (ctx->partials) cudaFree(ctx->partials);
   delete ctx;
+}
+
+int lossy_set_bursty(lossy_ctx* ctx, double p_enter_bad, double p_leave_bad, uint64_t* state) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (!state) {
+    ctx->burst_state = nullptr;
+    return LOSSY_OK;
+  }
+  if (!(p_enter_bad >= 0.0 && p_enter_bad < 1.0) || !(p_leave_bad > 0.0 && p_leave_bad <= 1.0))
+    return fail(ctx, LOSSY_EINVAL, "bursty loss: need 0 <= P(good->bad) < 1 and 0 < P(bad->good) <= 1");
+  if (ctx->K >= (1ull << 32)) return fail(ctx, LOSSY_EINVAL, "too many packets for bursty loss");
+  if (reinterpret_cast<uintptr_t>(state) & 7u) return fail(ctx, LOSSY_EINVAL, "state: misaligned");
+  ctx->burst_state = state;
+  ctx->Tenter = threshold_of(p_enter_bad);
+  ctx->Tstay = p_leave_bad >= 1.0 ? 0u : threshold_of(1.0 - p_leave_bad);
+  return LOSSY_OK;
 }
 
 int lossy_set_lr(lossy_ctx* ctx, float lr) {

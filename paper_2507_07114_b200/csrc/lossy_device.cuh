@@ -39,6 +39,8 @@ struct Params {
   uint64_t* stale_bits;   // optional output (BCAST)
   const uint8_t* count_in;  // STEP without AGG and ZERO_SKIP: received counts
   double* partials;       // DRIFT: [gridDim.x][kMaxW] per-block squared sums
+  const uint64_t* burst_in;  // bursty loss: link states after the previous step, [2][K] (row 0 gradient links, row 1 broadcast links)
+  uint64_t* burst_out;       // link states after this step, same layout (a different buffer)
   uint64_t n;
   uint64_t packet_base;
   uint64_t step_key;      // hash key of (seed, step), derived on the host
@@ -50,6 +52,8 @@ struct Params {
   uint32_t P;
   uint32_t W;
   uint32_t Tg, Tp;        // drop iff hash < T
+  uint32_t Tenter, Tstay; // bursty loss: a good link turns bad iff hash < Tenter, a bad one stays bad iff hash < Tstay
+  uint32_t K;             // packets in the bucket
   uint32_t flags;
   uint32_t prefetch_next; // register kernel: L2-prefetch the warp's next chunk
   float lr, b1, b2, omb1, omb2, ibc1, ibc2, eps;

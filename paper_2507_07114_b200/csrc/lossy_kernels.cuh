@@ -29,34 +29,62 @@ __device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8],
 
 // Delivery indicators of packet k (owner j), evaluated one worker per lane and gathered by ballot:
 // recv bit i = gradient piece of worker i reached the owner; stale bit i = replica i missed the broadcast.
+// Independent loss: one threshold compare per link. Bursty loss (P.burst_in set): each link is a two-state
+// chain on the same hash value, bad_t = bad_{t-1} ? (u < Tstay) : (u < Tenter), lost iff bad; the new states
+// come back in gbad / pbad for the one caller that stores them.
 template <int PH>
 __device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32_t j, int lane, uint64_t& recv,
-                                             uint64_t& stale) {
+                                             uint64_t& stale, uint64_t& gbad, uint64_t& pbad) {
   const uint32_t W = P.W;
   const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k);
   const uint32_t i0 = lane, i1 = lane + 32;
+  const bool bursty = P.burst_in != nullptr;
+  gbad = 0;
+  pbad = 0;
   if constexpr (PH & AGG) {
     // Algorithm 1's gradient half: the reduce is reliable and ONE draw (the owner's own link of the
     // hash) keeps or drops the packet's whole aggregate; otherwise one draw per contributing worker.
     const bool alg1 = P.ghat_prev != nullptr;
     const uint32_t src0 = alg1 ? j : i0, src1 = alg1 ? j : i1;
-    bool s0 = i0 < W && (pair_hash(pkey, src0, j) >= P.Tg || (!alg1 && (P.flags & 1u) && i0 == j));
-    uint32_t lo = __ballot_sync(0xFFFFFFFFu, s0), hi = 0;
+    const uint64_t gin = bursty ? P.burst_in[k] : 0ull;
+    const uint32_t u0 = pair_hash(pkey, src0, j);
+    const bool was0 = (gin >> (alg1 ? 0u : i0)) & 1ull;
+    bool lost0 = bursty ? (was0 ? u0 < P.Tstay : u0 < P.Tenter) : u0 < P.Tg;
+    if (!alg1 && (P.flags & 1u) && i0 == j) lost0 = false;
+    uint32_t lo = __ballot_sync(0xFFFFFFFFu, i0 < W && !lost0), hi = 0;
+    uint32_t blo = __ballot_sync(0xFFFFFFFFu, i0 < W && lost0), bhi = 0;
     if (W > 32) {
-      bool s1 = i1 < W && (pair_hash(pkey, src1, j) >= P.Tg || (!alg1 && (P.flags & 1u) && i1 == j));
-      hi = __ballot_sync(0xFFFFFFFFu, s1);
+      const uint32_t u1 = pair_hash(pkey, src1, j);
+      const bool was1 = (gin >> (alg1 ? 0u : i1)) & 1ull;
+      bool lost1 = bursty ? (was1 ? u1 < P.Tstay : u1 < P.Tenter) : u1 < P.Tg;
+      if (!alg1 && (P.flags & 1u) && i1 == j) lost1 = false;
+      hi = __ballot_sync(0xFFFFFFFFu, i1 < W && !lost1);
+      bhi = __ballot_sync(0xFFFFFFFFu, i1 < W && lost1);
     }
     recv = ((uint64_t)hi << 32) | lo;
+    gbad = alg1 ? (uint64_t)(blo & 1u) : (((uint64_t)bhi << 32) | blo);
   }
   if constexpr (PH & BCAST) {
-    bool d0 = i0 < W && i0 != j && pair_hash(pkey, j, i0) < P.Tp;
+    const uint64_t pin = bursty ? P.burst_in[(size_t)P.K + k] : 0ull;
+    const uint32_t u0 = pair_hash(pkey, j, i0);
+    const bool was0 = (pin >> i0) & 1ull;
+    const bool d0 = i0 < W && i0 != j && (bursty ? (was0 ? u0 < P.Tstay : u0 < P.Tenter) : u0 < P.Tp);
     uint32_t lo = __ballot_sync(0xFFFFFFFFu, d0), hi = 0;
     if (W > 32) {
-      bool d1 = i1 < W && i1 != j && pair_hash(pkey, j, i1) < P.Tp;
+      const uint32_t u1 = pair_hash(pkey, j, i1);
+      const bool was1 = (pin >> i1) & 1ull;
+      const bool d1 = i1 < W && i1 != j && (bursty ? (was1 ? u1 < P.Tstay : u1 < P.Tenter) : u1 < P.Tp);
       hi = __ballot_sync(0xFFFFFFFFu, d1);
     }
     stale = ((uint64_t)hi << 32) | lo;
+    pbad = stale;
   }
+}
+template <int PH>
+__device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32_t j, int lane, uint64_t& recv,
+                                             uint64_t& stale) {
+  uint64_t gbad, pbad;
+  packet_masks<PH>(P, k, j, lane, recv, stale, gbad, pbad);
 }
 
 template <int PH, class GT, class RT, int OPT>
@@ -79,8 +107,8 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
     if (in_pkt < P.P && e < P.n) nvalid = (P.n - e >= 8) ? 8 : (int)(P.n - e);
 
     // ---- delivery indicators of this packet (warp-uniform) -------------------
-    uint64_t recv = 0, stale = 0;
-    packet_masks<PH>(P, k, j, lane, recv, stale);
+    uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
+    packet_masks<PH>(P, k, j, lane, recv, stale, gbad, pbad);
     // Pull the NEXT chunk of this warp toward L2 while this one is processed. Worth its
     // instructions only when few workers feed a chunk (measured: +3..13 % for W <= 8, a loss above).
     if (P.prefetch_next) {
@@ -120,6 +148,10 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
       }
       if constexpr (PH & BCAST) {
         if (P.stale_bits) P.stale_bits[k] = stale;
+      }
+      if (P.burst_out) {   // the first chunk of a packet stores its links' new states
+        if constexpr (PH & AGG) P.burst_out[k] = gbad;
+        if constexpr (PH & BCAST) P.burst_out[(size_t)P.K + k] = pbad;
       }
     }
     // Lanes past a short packet or past the bucket end keep nvalid == 0: they stay in the

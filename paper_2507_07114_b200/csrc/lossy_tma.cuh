@@ -231,13 +231,17 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       const uint32_t j = k / P.pps;
       const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
       const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
-      uint64_t recv = 0, stale = 0;
-      packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale);
+      uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
+      packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale, gbad, pbad);
       const uint32_t cnt = __popcll(recv);
       if (c == 0 && lane == 0) {
         if (P.count) P.count[k] = (uint8_t)cnt;
         if (P.recv_bits) P.recv_bits[k] = recv;
         if (P.stale_bits) P.stale_bits[k] = stale;
+        if (P.burst_out) {   // bursty loss: the packet's first tile stores its links' new states
+          P.burst_out[k] = gbad;
+          P.burst_out[(size_t)P.K + k] = pbad;
+        }
       }
       if constexpr (DRIFTK) {
         for (uint32_t i = lane; i < W; i += 32)

@@ -62,8 +62,8 @@ class GpuRun:
     """State of one simulated run on the GPU, advanced through the C ABI."""
 
     def __init__(self, w: workload.Workload, *, flags=0, p_grad=None, p_param=None, theta0=None, device="cuda",
-                 alg1=False):
-        self.w, self.dev, self.alg1 = w, device, alg1
+                 alg1=False, burst=None):
+        self.w, self.dev, self.alg1, self.burst = w, device, alg1, burst
         self.ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems,
                                 p_grad=w.p if p_grad is None else p_grad,
                                 p_param=w.p if p_param is None else p_param, seed=w.seed,
@@ -83,6 +83,16 @@ class GpuRun:
         self.stale = torch.zeros(K, dtype=torch.int64, device=device)
         self.norms = torch.zeros(W, dtype=torch.float32, device=device)
         self.sumsq = torch.zeros(W, dtype=torch.float64, device=device)
+        self.burst_state = None
+        if burst is not None:
+            self.burst_state = torch.zeros(4 * K, dtype=torch.int64, device=device)   # [2 buffers][2 rows][K]
+            L.lossy_set_bursty(self.ctx, burst[0], burst[1], self.burst_state)
+
+    def burst_rows(self, t):
+        """Link states after step t as numpy [2][K] (row 0 gradient links, row 1 broadcast links)."""
+        K = self.w.K
+        buf = self.burst_state.view(2, 2, K)[t & 1]
+        return to_np(buf).view(np.uint64)
 
     def close(self):
         if self.ctx is not None:
@@ -129,14 +139,14 @@ class GpuRun:
 
 
 def make_oracle(w: workload.Workload, *, flags=0, p_grad=None, p_param=None, theta0=None, k0=0, n_slab=None,
-                e0=0, alg1=False):
+                e0=0, alg1=False, burst=None):
     n_slab = w.n - e0 if n_slab is None else n_slab
     th = workload.theta0_slab(w, e0, e0 + n_slab) if theta0 is None else theta0
     return O.Oracle(W=w.W, n=w.n, packet_elems=w.packet_elems, p_grad=w.p if p_grad is None else p_grad,
                     p_param=w.p if p_param is None else p_param, seed=w.seed, grad_dtype=odtype(w.grad_dtype),
                     replica_dtype=odtype(w.replica_dtype), optimizer=O.ADAM if w.optimizer == "adam" else O.SGD,
                     theta0=to_np(th), lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, flags=flags,
-                    packet_base=w.packet_base, k0=k0, n_slab=n_slab, alg1=alg1)
+                    packet_base=w.packet_base, k0=k0, n_slab=n_slab, alg1=alg1, burst=burst)
 
 
 def compare_state(gpu: GpuRun, orc, what, e0=0, e1=None):
@@ -160,10 +170,10 @@ def compare_outputs(out, ref, what, with_ghat=True):
 
 
 def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None, p_param=None, exact=True,
-               alg1=False):
+               alg1=False, burst=None):
     """Element-by-element parity of a whole (small) run. Returns the GpuRun for further checks."""
-    gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param, alg1=alg1)
-    orc = make_oracle(w, flags=flags & 3, p_grad=p_grad, p_param=p_param, alg1=alg1)   # bit 4 only picks the kernel
+    gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param, alg1=alg1, burst=burst)
+    orc = make_oracle(w, flags=flags & 3, p_grad=p_grad, p_param=p_param, alg1=alg1, burst=burst)   # bit 4 only picks the kernel
     for t in range(1, steps + 1):
         gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]
         gd = [g.cuda() for g in gs]
@@ -173,6 +183,8 @@ def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None,
         compare_state(gpu, orc, f"{w.name} step {t}")
         if alg1:
             assert_same(to_np(gpu.ghat_prev), orc.ghat_prev, f"{w.name} step {t} ghat_prev")
+        if burst is not None:
+            assert_same(gpu.burst_rows(t), orc.burst_state, f"{w.name} step {t} link states")
     L.lossy_device_status(gpu.ctx)      # raises if a bounded wait inside a kernel gave up
     if exact:
         # fixed order + separately rounded operations on both sides: the state is in fact bit-identical

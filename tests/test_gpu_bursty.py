@@ -1,0 +1,63 @@
+"""GPU parity of the bursty (two-state chain per link) loss against the oracle: masks, link states,
+counts and stale sets bit-exact, floats within the usual bar, on every kernel."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2507_07114_b200 as L
+import workload
+from parity_util import GpuRun, run_parity
+
+pytestmark = pytest.mark.gpu
+REG = L.LOSSY_REGISTER_PATH
+
+CASES = [
+    # name, W, n, P, (p_enter, p_leave), opt, gd, rd, flags, alg1
+    ("cfg2_shape", 8, 2048 * 37 + 1003, 2048, (0.05, 0.3), "adam", "bf16", "bf16", 0, False),
+    ("long_bursts", 8, 2048 * 40, 2048, (0.02, 0.08), "adam", "bf16", "bf16", 0, False),
+    ("memoryless", 6, 1024 * 30 + 64, 1024, (0.2, 0.8), "sgd", "f32", "f32", 0, False),
+    ("w64", 64, 4096 * 40, 4096, (0.05, 0.4), "adam", "bf16", "bf16", 0, False),
+    ("w40_self_lossless", 40, 1024 * 21, 1024, (0.3, 0.5), "sgd", "bf16", "f32", L.LOSSY_SELF_LOSSLESS, False),
+    ("small_packets", 5, 256 * 77 + 8, 256, (0.1, 0.2), "adam", "bf16", "bf16", 0, False),
+    ("always_leave", 4, 1024 * 12, 1024, (0.5, 1.0), "sgd", "f32", "bf16", 0, False),
+    ("alg1_one_chain_per_packet", 8, 2048 * 33, 2048, (0.1, 0.3), "adam", "bf16", "bf16", 0, True),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+@pytest.mark.parametrize("mode", ["fused", "fused_reg", "unfused"])
+def test_bursty_parity(case, mode):
+    name, W, n, P, burst, opt, gd, rd, flags, alg1 = case
+    w = workload.Workload("burst_" + name, W, n, P, 0.0, opt, 1e-2 if opt == "sgd" else 3e-4, gd, rd, 8, seed=31)
+    gpu, orc = run_parity(w, 8, fused=mode != "unfused", flags=flags | (REG if mode == "fused_reg" else 0),
+                          alg1=alg1, burst=burst)
+    assert int((gpu.count < W).sum()) > 0 and int(gpu.stale.ne(0).sum()) > 0
+
+
+def test_burstiness_shows_in_the_loss_runs_and_switching_back_works():
+    W, P, K = 8, 2048, 600
+    w = workload.Workload("burst_runs", W, P * K, P, 0.0, "sgd", 1e-2, "bf16", "bf16", 40, seed=2)
+    run = GpuRun(w, burst=(0.05, 0.25))
+    lost = []
+    for t in range(1, 41):
+        run.step_fused(t, [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(W)])
+        lost.append(~run.recv.cpu().numpy().view(np.uint64) & np.uint64(0xFF))
+    x = np.stack(lost)[10:]
+    bits = ((x[..., None] >> np.arange(8, dtype=np.uint64)) & np.uint64(1)).astype(np.float64)
+    rate = bits.mean()
+    assert abs(rate / (0.05 / 0.30) - 1) < 0.06
+    c = ((bits[1:] - rate) * (bits[:-1] - rate)).mean() / (rate * (1 - rate))
+    assert abs(c - 0.70) < 0.04                                   # lag-1 correlation 1 - p_enter - p_leave
+    L.lossy_set_bursty(run.ctx, 0.0, 1.0, None)                    # back to independent loss (p = 0 here)
+    run.step_fused(41, [workload.grad_slab(w, 41, i, 0, w.n, "cuda") for i in range(W)])
+    torch.cuda.synchronize()
+    assert int(run.count.min()) == W
+
+
+def test_bad_chain_arguments_are_rejected():
+    w = workload.Workload("burst_bad", 2, 2048, 1024, 0.0, "sgd", 1e-2, "f32", "f32", 1)
+    run = GpuRun(w)
+    st = torch.zeros(8, dtype=torch.int64, device="cuda")
+    for a, b in ((1.0, 0.5), (-0.1, 0.5), (0.1, 0.0), (0.1, 1.5)):
+        with pytest.raises(L.LossyError):
+            L.lossy_set_bursty(run.ctx, a, b, st)
