@@ -61,3 +61,30 @@ def test_bad_chain_arguments_are_rejected():
     for a, b in ((1.0, 0.5), (-0.1, 0.5), (0.1, 0.0), (0.1, 1.5)):
         with pytest.raises(L.LossyError):
             L.lossy_set_bursty(run.ctx, a, b, st)
+
+
+def test_drift_under_bursts_settles_at_sigma2_times_the_mean_age():
+    """The bounded-drift argument with correlated loss: for i.i.d. increments a replica's squared distance
+    from the owner is (elements it does not own) * sigma^2 * E[age], and the chain's mean age is
+    pi_bad / P(bad->good); it stays O(1) in t."""
+    from math import comb
+
+    W, a, b, lr, sg = 8, 0.1, 0.3, 1e-2, 1e-3
+    n = 1024 * 16000
+    w = workload.Workload("burst_drift", W, n, 1024, 0.0, "sgd", lr, "bf16", "f32", 90, grad_sigma=sg, seed=6)
+    run = GpuRun(w, burst=(a, b))
+    hist = []
+    for t in range(1, 91):
+        run.step_fused(t, [workload.grad_slab(w, t, i, 0, n, "cuda") for i in range(W)], outputs=False)
+        hist.append(run.norms.double().cpu().numpy() ** 2)
+    pi_b = a / (a + b)
+    q = 1 - pi_b
+    inv_c = sum(comb(W, c) * q ** c * pi_b ** (W - c) / c for c in range(1, W + 1))
+    sigma2 = (lr * sg) ** 2 * inv_c
+    pps = (w.K + W - 1) // W
+    own = np.array([min(w.K, (i + 1) * pps) - min(w.K, i * pps) for i in range(W)]) * 1024
+    want = (n - own) * sigma2 * pi_b / b
+    late = np.mean(hist[50:], axis=0)
+    assert np.all(np.abs(late / want - 1) < 0.05), late / want
+    # no growth with t (window means of ~13,000 packets with ages correlated over a few steps: ~1.2 % noise each)
+    assert np.all(np.abs(np.mean(hist[70:], axis=0) / np.mean(hist[50:70], axis=0) - 1) < 0.07)
