@@ -201,3 +201,39 @@ def test_empty_bucket_is_a_noop_and_bad_arguments_are_rejected():
         L.lossy_fused_step(ctx, 1, [mis, g[1]], th, th.clone(), th.clone(), r)
     assert L.lossy_kernel_launches(ctx) == 0            # nothing was launched for rejected calls
     L.lossy_destroy(ctx)
+
+
+@pytest.mark.parametrize("path_flag", [0, REG], ids=["bulk", "reg"])
+@pytest.mark.parametrize("opt", ["sgd", "adam"])
+def test_extreme_magnitudes_stay_bit_identical(path_flag, opt):
+    """Gradients spanning 2^-120 .. 2^100 (denormal sums, overflowing squares, infinities and the NaNs Adam
+    then produces): IEEE division, square root and the bf16 cast agree bit for bit on both sides."""
+    W, P, K = 5, 1024, 24
+    n = P * K
+    w = workload.Workload("extreme_" + opt, W, n, P, 0.2, opt, 1e-2 if opt == "sgd" else 3e-4, "bf16", "bf16", 4,
+                          seed=77)
+    gpu, orc = GpuRun(w, flags=path_flag), make_oracle(w)
+    gen = torch.Generator().manual_seed(5)
+    for t in range(1, 5):
+        gs = []
+        for i in range(W):
+            base = workload.grad_slab(w, t, i, 0, n).float()
+            expo = torch.randint(-120, 101, (n,), generator=gen)
+            gs.append((base * 1e3 * torch.pow(2.0, expo.float())).to(torch.bfloat16))
+        gpu.step_fused(t, [g.cuda() for g in gs])
+        orc.step(t, [to_np(g) for g in gs])
+        torch.cuda.synchronize()
+        for name, a, b in (("master", gpu.master, orc.master), ("m", gpu.m, orc.m), ("v", gpu.v, orc.v)):
+            if opt == "sgd" and name != "master":
+                continue
+            ga, gb = to_np(a).view(np.uint32), b.view(np.uint32)
+            nan_a, nan_b = np.isnan(to_np(a)), np.isnan(b)
+            assert np.array_equal(nan_a, nan_b), f"{name}: NaN positions differ at step {t}"
+            assert np.array_equal(ga[~nan_a], gb[~nan_b]), f"{name}: bits differ at step {t}"
+        for i in range(W):
+            ra, rb = to_np(gpu.replicas[i]), orc.replicas[i]
+            nan = (ra & 0x7FFF) > 0x7F80
+            assert np.array_equal(nan, (rb & 0x7FFF) > 0x7F80)
+            assert np.array_equal(ra[~nan], rb[~nan]), f"replica {i}: bits differ at step {t}"
+    if opt == "adam":
+        assert np.isnan(orc.master).any() or np.isinf(orc.v).any()      # the overflow paths were reached
