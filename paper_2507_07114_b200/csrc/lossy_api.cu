@@ -24,6 +24,8 @@ struct lossy_ctx {
   uint32_t max_blocks;   // capacity of `partials`
   double* partials;      // device, [max_blocks][kMaxW], followed by the status word
   uint32_t* status;      // device status word: 0 = fine, 1 = a bounded wait in a kernel gave up
+  uint32_t* ticket;      // device counter of finished blocks (last-block drift finalisation), zero between calls
+  bool plan_only;        // launch helpers only report their grid size
   uint64_t* burst_state; // bursty loss: caller-owned device array [2 buffers][2 rows][K], or NULL
   uint32_t Tenter, Tstay;
   int smem_optin;        // largest dynamic shared memory a block may opt in to
@@ -113,6 +115,16 @@ TmaPolicy tma_policy(const lossy_config& c) {
   return t;
 }
 
+constexpr int kMaxDevices = 64;
+
+// Dynamic shared memory one CTA of the bulk-copy kernel may use: the CTAs of one SM share 227 KB.
+template <int CW>
+uint32_t tma_smem_budget(const lossy_ctx* ctx) {
+  uint32_t budget = (227u * 1024u) / TmaShape<CW>::kCtasPerSm - 1024u;
+  if ((uint32_t)ctx->smem_optin < budget) budget = (uint32_t)ctx->smem_optin;
+  return budget;
+}
+
 template <int CW, int GS>
 bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   constexpr uint32_t kGroup = GS;
@@ -126,8 +138,7 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   G.groups = (c.W + kGroup - 1) / kGroup;
   uint32_t sb = G.grad_slots * kTile * gb + 3 * kTile * 4 + kTile * rb;
   G.stage_bytes = (sb + 127u) & ~127u;
-  uint32_t budget = (227u * 1024u) / TmaShape<CW>::kCtasPerSm - 1024u;   // the CTAs of one SM share 227 KB
-  if ((uint32_t)ctx->smem_optin < budget) budget = (uint32_t)ctx->smem_optin;
+  const uint32_t budget = tma_smem_budget<CW>(ctx);
   if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
   G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
   if (G.stages > (uint32_t)kMaxStages) G.stages = kMaxStages;
@@ -145,20 +156,22 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS>;
   constexpr int kThreadsTma = TmaShape<CW>::kThreads;
   const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
-  int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreadsTma, smem);
-  if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
-  if (per_sm < 1) per_sm = 1;
-  if (per_sm > TmaShape<CW>::kCtasPerSm) per_sm = TmaShape<CW>::kCtasPerSm;
-  uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
+  // launch bounds and the shared-memory budget guarantee kCtasPerSm resident CTAs per SM
+  uint32_t blocks = (uint32_t)(ctx->num_sms * TmaShape<CW>::kCtasPerSm);
   if (blocks > G.num_tiles) blocks = G.num_tiles;
+  *blocks_out = blocks;
+  if (ctx->plan_only) return LOSSY_OK;
+  static bool opted_in[kMaxDevices];   // per kernel instantiation and device: raise the dynamic shared memory limit once
+  cudaError_t e;
+  if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
+    if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
+    if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+  }
   kern<<<blocks, kThreadsTma, smem, s>>>(P, G);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda(ctx, "bulk-copy kernel launch", e);
   ctx->launches++;
-  *blocks_out = blocks;
   return LOSSY_OK;
 }
 
@@ -197,28 +210,26 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
 template <int PH, class GT, class RT, int OPT>
 int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out) {
   auto kern = lossy_kernel<PH, GT, RT, OPT>;
-  int per_sm = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, 0);
-  if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
-  if (per_sm < 1) per_sm = 1;
-  if (per_sm > kBlocksPerSmCap) per_sm = kBlocksPerSmCap;
+  static int occupancy[kMaxDevices];   // per kernel instantiation and device: resident blocks per SM
+  int per_sm = ctx->device < kMaxDevices ? occupancy[ctx->device] : 0;
+  cudaError_t e;
+  if (per_sm == 0) {
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, 0);
+    if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > kBlocksPerSmCap) per_sm = kBlocksPerSmCap;
+    if (ctx->device < kMaxDevices) occupancy[ctx->device] = per_sm;
+  }
   uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
   const uint32_t need = (P.num_chunks - P.chunk_begin + kWarps - 1) / kWarps;
   if (blocks > need) blocks = need;
   if (blocks > ctx->max_blocks - P.partials_row0) blocks = ctx->max_blocks - P.partials_row0;
   if (blocks == 0) blocks = 1;
+  if (blocks_out) *blocks_out = blocks;
+  if (ctx->plan_only) return LOSSY_OK;
   kern<<<blocks, kThreads, 0, s>>>(P);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda(ctx, "kernel launch", e);
-  ctx->launches++;
-  if (blocks_out) *blocks_out = blocks;
-  return LOSSY_OK;
-}
-
-int finalize_drift(lossy_ctx* ctx, uint32_t blocks, float* norms, double* sumsq, cudaStream_t s) {
-  drift_finalize_kernel<<<ctx->cfg.W, 32, 0, s>>>(ctx->partials, blocks, ctx->cfg.W, norms, sumsq);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return fail_cuda(ctx, "drift finalize launch", e);
   ctx->launches++;
   return LOSSY_OK;
 }
@@ -280,6 +291,7 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   e = cudaMalloc(&ctx->partials, pbytes + 256);
   if (e != cudaSuccess) { delete ctx; return e == cudaErrorMemoryAllocation ? LOSSY_ENOMEM : LOSSY_ECUDA; }
   ctx->status = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(ctx->partials) + pbytes);
+  ctx->ticket = ctx->status + 16;
   e = cudaMemset(ctx->status, 0, 256);
   if (e != cudaSuccess) { cudaFree(ctx->partials); delete ctx; return LOSSY_ECUDA; }
   *out = ctx;
@@ -398,9 +410,17 @@ int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas
   fill_common(ctx, 1, P);
   for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.replicas[i] = const_cast<void*>(replicas[i]);
   P.master = const_cast<float*>(master);
+  // grid size first, so that the kernel knows how many blocks will draw a ticket; the last one finalises
   uint32_t blocks = 0;
-  if (int rc = dispatch<DRIFT>(ctx, P, (cudaStream_t)stream, &blocks)) return rc;
-  return finalize_drift(ctx, blocks, norms, sumsq, (cudaStream_t)stream);
+  ctx->plan_only = true;
+  int rc = dispatch<DRIFT>(ctx, P, (cudaStream_t)stream, &blocks);
+  ctx->plan_only = false;
+  if (rc) return rc;
+  P.ticket = ctx->ticket;
+  P.total_rows = blocks;
+  P.norms = norms;
+  P.sumsq = sumsq;
+  return dispatch<DRIFT>(ctx, P, (cudaStream_t)stream, &blocks);
 }
 
 static int fused_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* master,
@@ -436,22 +456,37 @@ static int fused_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, f
   P.stale_bits = stale_bits;
   cudaStream_t s = (cudaStream_t)stream;
   const bool drift = norms || sumsq;
-  uint32_t rows = 0;
-  bool used_tma = false;
-  uint32_t tma_blocks = 0;
-  if (int rc = run_tma(ctx, P, drift, s, &tma_blocks, &used_tma)) return rc;
-  if (used_tma) {
-    // complete packets went through the bulk-copy pipeline; a short last packet takes the register kernel
-    rows = tma_blocks;
-    P.chunk_begin = (uint32_t)((ctx->cfg.n / ctx->cfg.packet_elems) * ctx->chunks_per_packet);
-    P.partials_row0 = rows;
+  // Complete packets go through the bulk-copy pipeline, a short last packet (or everything, when no
+  // bulk-copy build fits) through the register kernel. Pass 0 only sizes the grids: the blocks of both
+  // launches draw tickets from one counter and the last of them finalises the drift norms.
+  uint32_t tma_blocks = 0, tail_blocks = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    ctx->plan_only = pass == 0;
+    Params Q = P;
+    if (pass == 1 && drift) {
+      Q.ticket = ctx->ticket;
+      Q.total_rows = tma_blocks + tail_blocks;
+      Q.norms = norms;
+      Q.sumsq = sumsq;
+    }
+    bool used_tma = false;
+    int rc = run_tma(ctx, Q, drift, s, &tma_blocks, &used_tma);
+    if (!rc) {
+      if (used_tma) {
+        Q.chunk_begin = (uint32_t)((ctx->cfg.n / ctx->cfg.packet_elems) * ctx->chunks_per_packet);
+        Q.partials_row0 = tma_blocks;
+      } else {
+        tma_blocks = 0;
+      }
+      if (Q.chunk_begin < Q.num_chunks)
+        rc = drift ? dispatch<AGG | STEP | BCAST | DRIFT>(ctx, Q, s, &tail_blocks) : dispatch<AGG | STEP | BCAST>(ctx, Q, s, &tail_blocks);
+      else
+        tail_blocks = 0;
+    }
+    ctx->plan_only = false;
+    if (rc) return rc;
   }
-  if (P.chunk_begin < P.num_chunks) {
-    uint32_t blocks = 0;
-    if (int rc = drift ? dispatch<AGG | STEP | BCAST | DRIFT>(ctx, P, s, &blocks) : dispatch<AGG | STEP | BCAST>(ctx, P, s, &blocks)) return rc;
-    rows += blocks;
-  }
-  return drift ? finalize_drift(ctx, rows, norms, sumsq, s) : LOSSY_OK;
+  return LOSSY_OK;
 }
 
 int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* master, float* m, float* v,

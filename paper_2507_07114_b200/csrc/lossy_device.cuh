@@ -39,6 +39,12 @@ struct Params {
   uint64_t* stale_bits;   // optional output (BCAST)
   const uint8_t* count_in;  // STEP without AGG and ZERO_SKIP: received counts
   double* partials;       // DRIFT: [gridDim.x][kMaxW] per-block squared sums
+  // Drift finalisation inside the last block to finish (no second launch): `ticket` counts finished blocks
+  // over all launches of one call; NULL = a separate finalize kernel follows.
+  uint32_t* ticket;
+  uint32_t total_rows;    // partial rows (= blocks) of the whole call
+  float* norms;           // [W] or NULL
+  double* sumsq;          // [W], added to, or NULL
   const uint64_t* burst_in;  // bursty loss: link states after the previous step, [2][K] (row 0 gradient links, row 1 broadcast links)
   uint64_t* burst_out;       // link states after this step, same layout (a different buffer)
   uint64_t n;

@@ -27,6 +27,34 @@ __device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8],
   }
 }
 
+// Last-block drift finalisation. Every block has stored its row of `partials`; the block that draws the
+// last ticket sums the rows of each replica in a fixed order (lane l takes rows l, l+32, ..., then a shuffle
+// tree), so the result does not depend on which block happens to be last. Nothing here waits on another
+// block. Call with all threads of the block; `nwarps` warps share the replicas.
+__device__ __forceinline__ void drift_last_block(const Params& P, int warp, int lane, int nwarps) {
+  __shared__ uint32_t is_last;
+  __threadfence();                       // this block's partial row is visible device-wide ...
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t prev = atomicAdd(P.ticket, 1u);   // ... before its ticket is
+    is_last = prev + 1u == P.total_rows ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  for (uint32_t i = warp; i < P.W; i += nwarps) {
+    double t = 0.0;
+    for (uint32_t b = lane; b < P.total_rows; b += 32) t += __ldcg(&P.partials[(size_t)b * kMaxW + i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    if (lane == 0) {
+      if (P.sumsq) P.sumsq[i] += t;
+      if (P.norms) P.norms[i] = (float)sqrt(t);
+    }
+  }
+  if (threadIdx.x == 0) *P.ticket = 0u;  // ready for the next call on this context
+}
+
 // Delivery indicators of packet k (owner j), evaluated one worker per lane and gathered by ballot:
 // recv bit i = gradient piece of worker i reached the owner; stale bit i = replica i missed the broadcast.
 // Independent loss: one threshold compare per link. Bursty loss (P.burst_in set): each link is a two-state
@@ -300,6 +328,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
       for (int w = 0; w < kWarps; ++w) t += sh[w][threadIdx.x];
       P.partials[(size_t)(P.partials_row0 + blockIdx.x) * kMaxW + threadIdx.x] = t;
     }
+    if (P.ticket) drift_last_block(P, warp, lane, kWarps);
   }
 }
 

@@ -487,6 +487,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       for (int w = 0; w < kConsumerWarps; ++w) t += sh[w * kMaxW + threadIdx.x];
       P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
     }
+    if (P.ticket) drift_last_block(P, warp, lane, kConsumerWarps + 2);
   }
 }
 
