@@ -38,9 +38,9 @@ WORKLOAD = "cfg2_w8_layer_adam"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the fused kernel, from the ncu capture
-# summarised in profiles/fused_step_cfg2_w8_layer.md: 1769.7 MB on a 33,554,432-element cut of the
+# summarised in profiles/fused_step_cfg2_w8_layer.md: 1770.1 MB on a 33,554,432-element cut of the
 # workload, scaled by the elements processed (traffic is proportional to them).
-NCU_TRAFFIC_SMALL_CASE = (1769.7e6, 33554432)
+NCU_TRAFFIC_SMALL_CASE = (1770.1e6, 33554432)
 
 
 def algorithmic_bytes(w: workload.Workload, n: int | None = None) -> float:
@@ -330,7 +330,7 @@ def main():
                                      if pristine else None),
                          "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured"
                          else peak_src, "kernel": ("lossy_kernel<AGG|STEP|BCAST|DRIFT>" if args.register_path else "lossy_fused_tma_kernel")
-                         + " (+ W-warp drift finalize)",
+                         + " (drift norms finalised by its last block)",
                          "avg_launch_ms": avg_launch_ms, "min_launch_ms": min(per_launch_ms)},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
         }
