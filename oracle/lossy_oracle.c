@@ -332,3 +332,24 @@ int NAME(closed_loop_grads)(const oracle_config* c, uint64_t n_slab, const float
     }
   return 0;
 }
+
+/*
+ * The theorem's own quantity ("Quantifying Model Drift": D = theta^(i,j) - theta^(k,j) between two
+ * workers' copies): d2[i*W + k] += sum_e (replica_i[e] - replica_k[e])^2 for every pair, in double.
+ */
+int NAME(pairwise_sumsq)(const oracle_config* c, uint64_t n_slab, const void* const* replicas, double* d2) {
+  if (!c || !replicas || !d2) return 1;
+  const uint32_t W = c->W;
+  for (uint64_t e = 0; e < n_slab; ++e)
+    for (uint32_t i = 0; i < W; ++i) {
+      double ri = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[e])
+                                              : (double)((const float*)replicas[i])[e];
+      for (uint32_t k = 0; k < W; ++k) {
+        double rk = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[k])[e])
+                                                : (double)((const float*)replicas[k])[e];
+        double d = ri - rk;
+        d2[(size_t)i * W + k] += d * d;
+      }
+    }
+  return 0;
+}

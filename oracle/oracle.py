@@ -82,6 +82,9 @@ def _lib(f64: bool):
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
         ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
+        pw = getattr(lib, pre + "pairwise_sumsq")
+        pw.restype = C.c_int
+        pw.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p]
         cl = getattr(lib, pre + "closed_loop_grads")
         cl.restype = C.c_int
         cl.argtypes = [C.POINTER(OracleConfig), C.c_uint64] + [C.c_void_p] * 5
@@ -208,6 +211,16 @@ class Oracle:
         if rc != 0:
             raise ValueError("oracle_closed_loop_grads rejected its arguments")
         return out
+
+    def pairwise_sumsq(self):
+        """W x W matrix of sum_e (replica_i[e] - replica_k[e])^2, in double (the theorem's pairwise drift)."""
+        d2 = np.zeros((self.W, self.W), np.float64)
+        rt = _ptr_table(self.replicas)
+        rc = getattr(self.lib, self.pre + "pairwise_sumsq")(C.byref(self.cfg), self.n_slab, C.cast(rt, C.c_void_p),
+                                                            _ptr(d2))
+        if rc != 0:
+            raise ValueError("oracle_pairwise_sumsq rejected its arguments")
+        return d2
 
     def drift_sumsq(self):
         """Standalone drift: sum_e (replica_i[e] - cast(master[e]))^2 per replica, in double."""

@@ -158,3 +158,26 @@ def test_stale_fraction_is_binomial():
         trials = K - pps
         assert abs(stale_i - trials * p) < 4.5 * np.sqrt(trials * p * (1 - p))
     assert int(r["count"].sum()) == sum(bin(int(b)).count("1") for b in r["recv_bits"])
+
+
+def test_pairwise_drift_matrix_against_direct_sums_and_the_pair_constant():
+    """The theorem's own quantity between two receivers: symmetric, zero diagonal, equal to the direct
+    sum of squared differences, and stationary at 2p/(1-p^2) sigma^2 per element where neither owns."""
+    forms = _closed_forms()
+    W, K, P, p, T = 4, 4096, 4, 0.3, 160
+    o, rng, n = _run(W, K, P, p, 0, seed=12, p_grad=0.0)
+    acc, sig2 = [], []
+    keep = np.repeat(np.array([o.owner(k) not in (1, 2) for k in range(K)]), P)
+    for t in range(1, T + 1):
+        prev = o.master.copy()
+        o.step(t, [(rng.standard_normal(n) * 1e-1).astype(f32) for _ in range(W)])
+        if t > 40:
+            sig2.append(np.mean((o.master.astype(np.float64) - prev) ** 2))
+            d2 = o.pairwise_sumsq()
+            assert np.allclose(d2, d2.T, rtol=1e-14) and np.all(np.diag(d2) == 0)
+            R = np.stack([r.astype(np.float64) for r in o.replicas])
+            want = ((R[:, None, :] - R[None, :, :]) ** 2).sum(axis=2)
+            assert np.allclose(d2, want, rtol=1e-12)
+            # the part of D^2(1,2) over packets that neither 1 nor 2 owns
+            acc.append(np.sum((R[1] - R[2])[keep] ** 2) / keep.sum())
+    assert abs(np.mean(acc) / (np.mean(sig2) * forms[p][1]) - 1) < 0.04
