@@ -174,6 +174,18 @@ int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas
                 float* norms, double* sumsq, void* stream);
 
 /*
+ * drift_pairwise — the theorem's own quantity ("Quantifying Model Drift":
+ * D = theta^(i,j) - theta^(k,j) between two workers' copies): for every pair
+ *     d2[i*W + k] += sum_e ( float(replica_i[e]) - float(replica_k[e]) )^2 .
+ * A diagnostic: it re-reads each replica once per block of four partner
+ * replicas and is not part of the timed step.
+ *   d2   [W*W] fp64 device, ADDED to (zero it first; symmetric, zero diagonal)
+ * The sum over thread blocks uses fp64 atomics, so its order is not fixed: two
+ * runs agree to about 1e-15 relative, not bit for bit.
+ */
+int drift_pairwise(lossy_ctx* ctx, const void* const* replicas, double* d2, void* stream);
+
+/*
  * drift_norms_static — the same norms as drift_norms for callers that must not
  * allocate device memory. The paper has no counterpart: this entry point exists
  * only for the way the library is embedded.

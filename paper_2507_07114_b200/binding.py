@@ -21,7 +21,7 @@ LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_aggregate", "lossy_step", "lossy_broadcast",
-    "drift_norms", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
+    "drift_norms", "drift_pairwise", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
 
@@ -72,6 +72,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_broadcast.argtypes = [vp, u64, vp, vp, vp, vp]
     lib.drift_norms.restype = C.c_int
     lib.drift_norms.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.drift_pairwise.restype = C.c_int
+    lib.drift_pairwise.argtypes = [vp, vp, vp, vp]
     lib.drift_norms_static.restype = C.c_int
     lib.drift_norms_static.argtypes = [C.POINTER(lossy_config), vp, vp, vp, vp, vp]
     lib.lossy_fused_step.restype = C.c_int
@@ -172,6 +174,11 @@ def lossy_broadcast(ctx, step, master, replicas, stale_bits=None):
 
 def drift_norms(ctx, master, replicas, norms=None, sumsq=None):
     _check(ctx, load_library().drift_norms(ctx, _p(master), _table(replicas), _p(norms), _p(sumsq), _stream()))
+
+
+def drift_pairwise(ctx, replicas, d2):
+    """d2: fp64 device tensor of W*W elements, added to (zero it first)."""
+    _check(ctx, load_library().drift_pairwise(ctx, _table(replicas), _p(d2), _stream()))
 
 
 def drift_norms_static(*, W, n, packet_elems, replica_dtype, master, replicas, norms=None, sumsq=None):

@@ -506,6 +506,33 @@ int lossy_fused_step_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grad
                     sumsq, stream);
 }
 
+int drift_pairwise(lossy_ctx* ctx, const void* const* replicas, double* d2, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (!d2) return fail(ctx, LOSSY_EINVAL, "d2: NULL");
+  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  PairwiseArgs A;
+  memset(&A, 0, sizeof A);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) A.replicas[i] = replicas[i];
+  A.d2 = d2;
+  A.n = ctx->cfg.n;
+  A.W = ctx->cfg.W;
+  A.nblk = (ctx->cfg.W + 3) / 4;
+  const uint32_t pairs = A.nblk * (A.nblk + 1) / 2;
+  const uint64_t nvec = (A.n + 7) / 8;
+  uint64_t bx = (nvec + 255) / 256;
+  const uint64_t cap = (uint64_t)ctx->num_sms * 4;
+  if (bx > cap) bx = cap;
+  const dim3 grid((uint32_t)bx, pairs);
+  cudaStream_t s = (cudaStream_t)stream;
+  if (ctx->cfg.replica_dtype == LOSSY_BF16) drift_pairwise_kernel<BF16><<<grid, 256, 0, s>>>(A);
+  else drift_pairwise_kernel<F32><<<grid, 256, 0, s>>>(A);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "pairwise drift launch", e);
+  ctx->launches++;
+  return LOSSY_OK;
+}
+
 int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* target, const void* const* noise,
                             const void* const* replicas, void* const* grads_out, void* stream) {
   if (!ctx) return LOSSY_EINVAL;

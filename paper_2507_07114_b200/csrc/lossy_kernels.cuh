@@ -348,6 +348,75 @@ static __global__ void drift_finalize_kernel(const double* __restrict__ partials
   }
 }
 
+// Pairwise drift, the theorem's own quantity: d2[i*W + k] += sum_e (replica_i[e] - replica_k[e])^2.
+// blockIdx.y picks a pair of 4-replica blocks (I <= J); each lane keeps the 16 pair sums of its elements in
+// fp64 and walks 8-element vectors grid-stride in x. Cross-block accumulation uses fp64 atomics, so the order
+// of that last sum is not fixed (results agree to ~1e-15 relative). A diagnostic, not on the timed path.
+struct PairwiseArgs {
+  const void* replicas[kMaxW];
+  double* d2;
+  uint64_t n;
+  uint32_t W;
+  uint32_t nblk;   // ceil(W / 4)
+};
+
+template <class RT>
+static __global__ void __launch_bounds__(256) drift_pairwise_kernel(const __grid_constant__ PairwiseArgs A) {
+  // blockIdx.y -> (I, J) with I <= J
+  uint32_t I = 0, rem = blockIdx.y;
+  while (rem >= A.nblk - I) { rem -= A.nblk - I; ++I; }
+  const uint32_t J = I + rem;
+  double acc[16];
+#pragma unroll
+  for (int q = 0; q < 16; ++q) acc[q] = 0.0;
+  const uint64_t nvec = (A.n + 7) / 8;
+  for (uint64_t vi = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t e = vi * 8;
+    const int nvalid = A.n - e >= 8 ? 8 : (int)(A.n - e);
+    float a[4][8], b[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t ia = I * 4 + u, ib = J * 4 + u;
+      if (ia < A.W) widen<RT>(load8_any<RT>(A.replicas[ia], e, nvalid), a[u]);
+      if (ib < A.W) widen<RT>(load8_any<RT>(A.replicas[ib], e, nvalid), b[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        if (I * 4 + u < A.W && J * 4 + v < A.W) {
+          float s = 0.0f;
+#pragma unroll
+          for (int x = 0; x < 8; ++x) {
+            const float d = x < nvalid ? __fsub_rn(a[u][x], b[v][x]) : 0.0f;
+            s = __fadd_rn(s, __fmul_rn(d, d));
+          }
+          acc[u * 4 + v] += (double)s;
+        }
+      }
+  }
+  __shared__ double sh[8][16];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int q = 0; q < 16; ++q) {
+    double t = acc[q];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    if (lane == 0) sh[warp][q] = t;
+  }
+  __syncthreads();
+  if (threadIdx.x < 16) {
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += sh[w][threadIdx.x];
+    const uint32_t i = I * 4 + threadIdx.x / 4, k = J * 4 + threadIdx.x % 4;
+    if (i < A.W && k < A.W) {
+      atomicAdd(&A.d2[(size_t)i * A.W + k], t);
+      if (I != J) atomicAdd(&A.d2[(size_t)k * A.W + i], t);   // mirror; a diagonal block already holds both orders
+    }
+  }
+}
+
 // Closed-loop stand-in for the local gradient computation (Section 3 step (1)): worker i's gradient of
 // 1/2 sum a (theta - x*)^2 at ITS OWN replica plus its noise, g_i = cast(a * (replica_i - x*) + noise_i),
 // each operation rounded on its own. One lane per 8 elements, workers four at a time.

@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def _declared():
     text = open(os.path.join(ROOT, "include", "lossy.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(lossy_[a-z0-9_]+|drift_norms[a-z_]*)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(lossy_[a-z0-9_]+|drift_[a-z_]+)\s*\(", text)))
 
 
 def test_header_symbols_are_exported_and_bound():
