@@ -27,6 +27,8 @@
  *     `packet_elems` contiguous elements (the last may be short). Shard j, owned
  *     by worker j, is the contiguous packet range [j*pps, min(K,(j+1)*pps)) with
  *     pps = ceil(K / W)  (Section 3: theta = (theta^(1) ... theta^(N))).
+ *   - Packets evolve independently of one another, so a bucket may be split into packet
+ *     ranges run by different contexts (or GPUs): see shard_packet0 / bucket_packets.
  *   - Packet k of the bucket has the global packet id packet_base + k; only the
  *     drop-mask hash sees the global id, so a model can be streamed bucket by
  *     bucket with independent masks.
@@ -74,6 +76,13 @@ typedef struct {
   uint32_t optimizer;    /* LOSSY_SGD or LOSSY_ADAM                                     */
   uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH */
   float lr, beta1, beta2, eps; /* eta_t and Adam's constants (beta/eps unused for SGD)  */
+  /* Packet-range sharding (several GPUs simulate one bucket, each a contiguous range of its
+   * packets for all W workers): this context's packet 0 is packet shard_packet0 of a bucket of
+   * bucket_packets packets; owners and hash ids follow the whole bucket, `n` and every array
+   * are the range's. Both 0 = the context covers the whole bucket. A range may be ragged (n not
+   * a multiple of packet_elems) only if it ends the bucket. */
+  uint64_t shard_packet0;
+  uint64_t bucket_packets;
 } lossy_config;
 
 /*

@@ -5,4 +5,4 @@ from .binding import (EXPORTS, LossyError, drift_norms, drift_norms_static, drif
                       lossy_config, lossy_destroy, lossy_device_status, lossy_fused_step, lossy_fused_step_alg1, lossy_fused_step_host, lossy_hash_u32,
                       lossy_init, lossy_kernel_launches, lossy_last_error, lossy_mask, lossy_mask_grid, lossy_num_packets,
                       lossy_set_bursty, lossy_set_lr, lossy_step)
-from .sharding import shard_range  # noqa: F401
+from .sharding import packet_range_config, shard_range  # noqa: F401

@@ -32,7 +32,7 @@ class lossy_config(C.Structure):
         ("p_grad", C.c_double), ("p_param", C.c_double), ("seed", C.c_uint64),
         ("grad_dtype", C.c_uint32), ("replica_dtype", C.c_uint32), ("optimizer", C.c_uint32),
         ("flags", C.c_uint32), ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
-        ("eps", C.c_float),
+        ("eps", C.c_float), ("shard_packet0", C.c_uint64), ("bucket_packets", C.c_uint64),
     ]
 
 
@@ -131,13 +131,13 @@ def _check(ctx, rc):
 
 
 def lossy_init(*, W, n, packet_elems, p_grad, p_param, seed, grad_dtype, replica_dtype, optimizer, lr,
-               beta1=0.9, beta2=0.95, eps=1e-8, flags=0, packet_base=0):
+               beta1=0.9, beta2=0.95, eps=1e-8, flags=0, packet_base=0, shard_packet0=0, bucket_packets=0):
     """Create a context on the current CUDA device; returns an opaque handle (free with lossy_destroy)."""
     lib = load_library()
     torch.cuda.init()
     opt = {"sgd": LOSSY_SGD, "adam": LOSSY_ADAM}.get(optimizer, optimizer)
     cfg = lossy_config(W, packet_elems, n, packet_base, p_grad, p_param, seed, _dt(grad_dtype), _dt(replica_dtype),
-                       opt, flags, lr, beta1, beta2, eps)
+                       opt, flags, lr, beta1, beta2, eps, shard_packet0, bucket_packets)
     ctx = C.c_void_p()
     with torch.cuda.device(torch.cuda.current_device()):
         rc = lib.lossy_init(C.byref(cfg), C.byref(ctx))
@@ -186,7 +186,7 @@ def drift_norms_static(*, W, n, packet_elems, replica_dtype, master, replicas, n
 
     Raises LossyError with code LOSSY_ELIMIT when a size is beyond the static scratch's limits."""
     cfg = lossy_config(W, packet_elems, n, 0, 0.0, 0.0, 0, LOSSY_F32, _dt(replica_dtype), LOSSY_SGD, 0,
-                       0.0, 0.0, 0.0, 0.0)
+                       0.0, 0.0, 0.0, 0.0, 0, 0)
     rc = load_library().drift_norms_static(C.byref(cfg), _p(master), _table(replicas), _p(norms), _p(sumsq),
                                            _stream())
     if rc != LOSSY_OK:

@@ -60,7 +60,8 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   memset(&P, 0, sizeof P);
   const lossy_config& c = ctx->cfg;
   P.n = c.n;
-  P.packet_base = c.packet_base;
+  P.packet_base = c.packet_base + c.shard_packet0;   // the hash sees the global id of every packet
+  P.k0 = (uint32_t)c.shard_packet0;
   P.step_key = step_key_of(c.seed, step);
   P.num_chunks = ctx->num_chunks;
   P.chunks_per_packet = ctx->chunks_per_packet;
@@ -269,6 +270,13 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
   const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;
   if (K * cpp >= (1ull << 31)) return LOSSY_EINVAL;  // stream larger models bucket by bucket
+  if (cfg->bucket_packets) {
+    // a packet range of a larger bucket: inside it, and ragged only where the bucket ends
+    if (cfg->bucket_packets >= (1ull << 31) || cfg->shard_packet0 + K > cfg->bucket_packets) return LOSSY_EINVAL;
+    if (cfg->n % cfg->packet_elems != 0 && cfg->shard_packet0 + K != cfg->bucket_packets) return LOSSY_EINVAL;
+  } else if (cfg->shard_packet0) {
+    return LOSSY_EINVAL;
+  }
 
   lossy_ctx* ctx = new (std::nothrow) lossy_ctx;
   if (!ctx) return LOSSY_ENOMEM;
@@ -277,7 +285,9 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   ctx->K = K;
   ctx->chunks_per_packet = (uint32_t)cpp;
   ctx->num_chunks = (uint32_t)(K * cpp);
-  const uint64_t pps = (K + cfg->W - 1) / cfg->W;
+  // shard map of the WHOLE bucket: this context may cover only the packet range starting at shard_packet0
+  const uint64_t Kb = cfg->bucket_packets ? cfg->bucket_packets : K;
+  const uint64_t pps = (Kb + cfg->W - 1) / cfg->W;
   ctx->pps = pps ? (uint32_t)pps : 1u;
   ctx->Tg = threshold_of(cfg->p_grad);
   ctx->Tp = threshold_of(cfg->p_param);

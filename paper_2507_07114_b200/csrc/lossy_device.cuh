@@ -54,7 +54,8 @@ struct Params {
   uint32_t chunk_begin;   // first chunk this launch covers (a bulk-copy launch may own the chunks before it)
   uint32_t partials_row0; // first row of `partials` this launch writes
   uint32_t chunks_per_packet;
-  uint32_t pps;           // packets per shard
+  uint32_t pps;           // packets per shard (of the whole bucket)
+  uint32_t k0;            // bucket packet index of this context's packet 0 (a context may cover a packet range)
   uint32_t P;
   uint32_t W;
   uint32_t Tg, Tp;        // drop iff hash < T

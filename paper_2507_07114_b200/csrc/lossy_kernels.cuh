@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
   for (uint32_t q = P.chunk_begin + blockIdx.x * kWarps + warp; q < P.num_chunks; q += warps_in_grid) {
     const uint32_t k = q / P.chunks_per_packet;
     const uint32_t c = q - k * P.chunks_per_packet;
-    const uint32_t j = k / P.pps;  // owner W_j of packet k
+    const uint32_t j = (P.k0 + k) / P.pps;  // owner W_j of packet k
     const uint32_t in_pkt = c * kChunk + lane * 8;
     const uint64_t e = (uint64_t)k * P.P + in_pkt;
     int nvalid = 0;
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
         const uint32_t inn = cn * kChunk + lane * 8;
         const uint64_t en = (uint64_t)kn * P.P + inn;
         uint64_t rn = 0, sn = 0;
-        packet_masks<PH>(P, kn, kn / P.pps, lane, rn, sn);
+        packet_masks<PH>(P, kn, (P.k0 + kn) / P.pps, lane, rn, sn);
         if (inn < P.P && en + 8 <= P.n) {
           if constexpr (PH & (STEP | BCAST | DRIFT)) prefetch_l2(P.master + en);
           if constexpr ((PH & STEP) && OPT == 1) { prefetch_l2(P.m + en); prefetch_l2(P.v + en); }

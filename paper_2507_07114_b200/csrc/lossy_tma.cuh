@@ -228,7 +228,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
       const uint32_t k = tile / G.tiles_per_packet;
       const uint32_t c = tile - k * G.tiles_per_packet;
-      const uint32_t j = k / P.pps;
+      const uint32_t j = (P.k0 + k) / P.pps;
       const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
       const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
       uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;

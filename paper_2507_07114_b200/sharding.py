@@ -14,3 +14,15 @@ def shard_range(units: int, rank: int, world: int) -> tuple[int, int]:
     base, extra = divmod(units, world)
     lo = rank * base + min(rank, extra)
     return lo, lo + base + (1 if rank < extra else 0)
+
+
+def packet_range_config(total_elems: int, packet_elems: int, rank: int, world: int) -> dict:
+    """One bucket simulated by `world` GPUs, each a contiguous packet range for all W workers.
+
+    Returns the keyword arguments that describe rank's range to lossy_init (`n`, `shard_packet0`,
+    `bucket_packets`) plus the element offset `e0` of the range inside the bucket's arrays.
+    """
+    K = (total_elems + packet_elems - 1) // packet_elems
+    lo, hi = shard_range(K, rank, world)
+    e0, e1 = lo * packet_elems, min(total_elems, hi * packet_elems)
+    return {"n": e1 - e0, "shard_packet0": lo, "bucket_packets": K, "e0": e0}

@@ -31,8 +31,9 @@ def test_header_symbols_are_exported_and_bound():
 
 
 def test_config_struct_layout_matches_the_header():
-    # uint32 W, P; uint64 n, base; double x2; uint64 seed; uint32 x4; float x4
-    assert ctypes.sizeof(L.lossy_config) == 4 + 4 + 8 + 8 + 8 + 8 + 8 + 16 + 16
+    # uint32 W, P; uint64 n, base; double x2; uint64 seed; uint32 x4; float x4; uint64 x2
+    assert ctypes.sizeof(L.lossy_config) == 4 + 4 + 8 + 8 + 8 + 8 + 8 + 16 + 16 + 8 + 8
+    assert L.lossy_config.shard_packet0.offset == 80
     assert L.lossy_config.n.offset == 8 and L.lossy_config.seed.offset == 40 and L.lossy_config.lr.offset == 64
 
 

@@ -9,7 +9,7 @@ import torch.distributed as dist
 import torch.multiprocessing as mp
 
 import workload
-from paper_2507_07114_b200.sharding import shard_range
+from paper_2507_07114_b200.sharding import packet_range_config, shard_range
 from parity_util import make_oracle, to_np
 
 
@@ -21,6 +21,18 @@ def test_shard_range_partitions_exactly():
             assert all(a[1] == b[0] for a, b in zip(got[:-1], got[1:]))
             sizes = [b - a for a, b in got]
             assert max(sizes) - min(sizes) <= 1
+
+
+def test_packet_ranges_tile_the_bucket():
+    for n, P in ((2048 * 37 + 1003, 2048), (1024 * 11, 1024), (100, 256)):
+        K = (n + P - 1) // P
+        for world in (1, 2, 3, 8):
+            cfgs = [packet_range_config(n, P, r, world) for r in range(world)]
+            assert cfgs[0]["e0"] == 0 and sum(c["n"] for c in cfgs) == n
+            for a, b in zip(cfgs[:-1], cfgs[1:]):
+                assert a["e0"] + a["n"] == b["e0"] and a["n"] % P == 0      # only the last range may be ragged
+                assert b["shard_packet0"] * P == b["e0"]
+            assert all(c["bucket_packets"] == K for c in cfgs)
 
 
 BUCKETS = [512 * 9, 512 * 7 + 40, 512 * 12, 512 * 5, 512 * 3 + 8]
