@@ -24,5 +24,5 @@ def packet_range_config(total_elems: int, packet_elems: int, rank: int, world: i
     """
     K = (total_elems + packet_elems - 1) // packet_elems
     lo, hi = shard_range(K, rank, world)
-    e0, e1 = lo * packet_elems, min(total_elems, hi * packet_elems)
+    e0, e1 = min(total_elems, lo * packet_elems), min(total_elems, hi * packet_elems)   # a rank may get nothing
     return {"n": e1 - e0, "shard_packet0": lo, "bucket_packets": K, "e0": e0}
