@@ -158,6 +158,10 @@ def main():
     ap.add_argument("--p", type=float, default=None, help="override the drop probability")
     ap.add_argument("--workers", type=int, default=0, help="override W")
     ap.add_argument("--packet-elems", type=int, default=0, help="override the packet size")
+    ap.add_argument("--strong", action="store_true",
+                    help="N > 1: split ONE bucket into packet ranges, one per rank (default: one bucket per rank)")
+    ap.add_argument("--range", default="", metavar="R/G",
+                    help="single process: run only packet range R of G of the bucket (what rank R of a G-GPU --strong job runs)")
     ap.add_argument("--register-path", action="store_true", help="time the register-path kernel, not the bulk-copy pipeline")
     ap.add_argument("--e2e-steps", type=int, default=-1, help="steps of the host-buffer leg (default: min(steps, 10))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -185,7 +189,7 @@ def main():
     warmup = max(3, args.warmup)
     # the stored ncu traffic figure belongs to the unmodified default workload on the default kernel
     pristine = (args.workload == WORKLOAD and args.p is None and not args.workers and not args.packet_elems
-                and not args.register_path)
+                and not args.register_path and not args.range)
 
     if args.impl == "reference":
         if rank != 0:
@@ -213,22 +217,31 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
-    # every rank simulates its own bucket: global packet ids continue across ranks
-    w = workload.scaled(w, w.n, packet_base=rank * w.K, seed=w.seed)
+    full_n, e_off, rng_kw = w.n, 0, {}
+    if (args.strong and world > 1) or args.range:
+        # strong scaling: the ranks share one bucket, each a contiguous packet range for all W workers
+        r_, g_ = (int(x) for x in args.range.split("/")) if args.range else (rank, world)
+        pr = L.packet_range_config(w.n, w.packet_elems, r_, g_)
+        e_off = pr["e0"]
+        rng_kw = {"shard_packet0": pr["shard_packet0"], "bucket_packets": pr["bucket_packets"]}
+        w = workload.scaled(w, pr["n"])
+    else:
+        # weak scaling: every rank simulates its own bucket; global packet ids continue across ranks
+        w = workload.scaled(w, w.n, packet_base=rank * w.K, seed=w.seed)
     gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
     rdt = torch.bfloat16 if w.replica_dtype == "bf16" else torch.float32
     adam = w.optimizer == "adam"
     ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems, p_grad=w.p, p_param=w.p, seed=w.seed,
                        grad_dtype=gdt, replica_dtype=rdt, optimizer=w.optimizer, lr=w.lr, beta1=w.beta1,
                        beta2=w.beta2, eps=w.eps, packet_base=w.packet_base,
-                       flags=L.LOSSY_REGISTER_PATH if args.register_path else 0)
-    master = workload.theta0_slab(w, 0, w.n, dev)
+                       flags=L.LOSSY_REGISTER_PATH if args.register_path else 0, **rng_kw)
+    master = workload.theta0_slab(w, e_off, e_off + w.n, dev)
     m = torch.zeros_like(master) if adam else None
     v = torch.zeros_like(master) if adam else None
     replicas = [master.to(rdt) for _ in range(w.W)]
     norms = torch.zeros(w.W, dtype=torch.float32, device=dev)
     sumsq = torch.zeros(w.W, dtype=torch.float64, device=dev)
-    grad_sets = [gen_grads(w, s, dev) for s in (1, 2)]      # 2 sets, each larger than L2, used alternately
+    grad_sets = [gen_grads(w, s, dev, e_off, e_off + w.n) for s in (1, 2)]   # 2 sets, each larger than L2, alternate
     stream = torch.cuda.current_stream()
 
     def one_step(t):
@@ -268,8 +281,10 @@ def main():
     if dist is not None:
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
     total_ms = float(tmax.item())
-    B = algorithmic_bytes(w)
-    value = B * args.steps * world / (total_ms * 1e-3) / 1e9
+    B = algorithmic_bytes(w)                                  # this rank's bytes per step
+    strong = args.strong and world > 1
+    B_job = algorithmic_bytes(w, full_n) if strong else B * world
+    value = B_job * args.steps / (total_ms * 1e-3) / 1e9
     peak, peak_src = measured_peak()
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
     achieved = B / (avg_launch_ms * 1e-3) / 1e9
@@ -298,7 +313,7 @@ def main():
         if dist is not None:
             dist.all_reduce(tm, op=dist.ReduceOp.MAX)
         e2e_ms = float(tm.item())
-        e2e = {"value": B * e2e_steps * world / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+        e2e = {"value": B_job * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                "h2d_bytes_per_step": sum(g.numel() * g.element_size() for g in host_grads),
                "d2h_bytes_per_step": host_norms.numel() * 4, "steps": e2e_steps,
                "ms_per_step": e2e_ms / e2e_steps,
@@ -314,13 +329,15 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-            "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "strong" if strong else "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "steps_per_s": args.steps * world / (total_ms * 1e-3),
+            "steps_per_s": args.steps * (1 if strong else world) / (total_ms * 1e-3),
             "pct_of_hbm_peak": 100.0 * value / world / peak,
             "config": {"workload": w.name, "W": w.W, "n": w.n, "packet_elems": w.packet_elems, "p": w.p,
                        "optimizer": w.optimizer, "grad_dtype": w.grad_dtype, "replica_dtype": w.replica_dtype,
-                       "bytes_per_step": B, "parallelism": f"{world} independent bucket(s), one per GPU",
+                       "bytes_per_step": B, "parallelism": (f"one bucket in {world} packet ranges, one per GPU" if strong
+                                       else f"{world} independent bucket(s), one per GPU"),
                        "l2": "no flush: each step streams %.1f GB of state, far larger than the 126 MB L2; "
                              "two gradient sets alternate" % (B / 1e9),
                        "drift_norm_max_last_step": final_norm_max},
