@@ -35,7 +35,7 @@ def algorithmic_bytes(w, alg1=False):
     return b + (4 * w.n if alg1 else 0)
 
 
-def run_point(w, steps, warmup=3, grad_sets=2, alg1=False):
+def run_point(w, steps, warmup=3, grad_sets=2, alg1=False, graph=False):
     dev = torch.device("cuda")
     gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
     rdt = torch.bfloat16 if w.replica_dtype == "bf16" else torch.float32
@@ -74,10 +74,31 @@ def run_point(w, steps, warmup=3, grad_sets=2, alg1=False):
     torch.cuda.synchronize()
     L.lossy_device_status(ctx)
     ms = e0.elapsed_time(e1) / steps
+    graph_sps = None
+    if graph:
+        # launch-bound case: capture `steps` consecutive steps once, replay them as one graph launch
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(steps):
+                    step(t + 1 + i)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        reps = 20
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        graph_sps = reps * steps / (e0.elapsed_time(e1) * 1e-3)
+        L.lossy_device_status(ctx)
     L.lossy_destroy(ctx)
     gbs = algorithmic_bytes(w, alg1) / (ms * 1e-3) / 1e9
     return {"workload": w.name + ("[alg1]" if alg1 else ""), "W": w.W, "P": w.packet_elems, "p": w.p, "ms_per_step": ms, "GBps": gbs,
-            "frac_of_measured_peak": gbs / _peak(), "steps_per_s": 1e3 / ms, "max_drift_norm": float(worst.max())}
+            "frac_of_measured_peak": gbs / _peak(), "steps_per_s": 1e3 / ms, "max_drift_norm": float(worst.max()),
+            **({"steps_per_s_cuda_graph": graph_sps} if graph_sps else {})}
 
 
 def main():
@@ -100,7 +121,7 @@ def main():
                 points.append(workload.scaled(cfg["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=P, p=p,
                                               name=f"cfg5_w16_P{P}_p{p}"))
     for w in points:
-        r = run_point(w, args.steps or w.steps, grad_sets=1 if w.W >= 64 else 2)
+        r = run_point(w, args.steps or w.steps, grad_sets=1 if w.W >= 64 else 2, graph=w.n <= (1 << 22))
         print(json.dumps(r), flush=True)
     if "alg1" in want:
         # Algorithm 1 mode on the config-2 bucket: packet-granular and shard-granular (P = n / W) drops

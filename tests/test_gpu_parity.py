@@ -237,3 +237,33 @@ def test_extreme_magnitudes_stay_bit_identical(path_flag, opt):
             assert np.array_equal(ra[~nan], rb[~nan]), f"replica {i}: bits differ at step {t}"
     if opt == "adam":
         assert np.isnan(orc.master).any() or np.isinf(orc.v).any()      # the overflow paths were reached
+
+
+def test_ten_steps_captured_in_a_cuda_graph_replay_bit_identically():
+    """The calls are stream-asynchronous and synchronise nothing, so a launch-bound loop (config 1: 40 MB per
+    step) can be captured once and replayed as one graph launch."""
+    w = CFG["cfg1_w4_sgd_f32"]
+    eager, graphed = GpuRun(w), GpuRun(w)
+    grads = [[workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)] for t in range(1, 11)]
+    for t in range(1, 11):
+        eager.step_fused(t, grads[t - 1], outputs=False)
+    saved = [graphed.master.clone()] + [r.clone() for r in graphed.replicas]
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graphed.step_fused(1, grads[0], outputs=False)          # first use outside capture (one-time set-up)
+        for dst, src in zip([graphed.master] + graphed.replicas, saved):
+            dst.copy_(src)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for t in range(1, 11):
+                graphed.step_fused(t, grads[t - 1], outputs=False)
+    for _ in range(2):                                           # replay twice from the same start
+        for dst, src in zip([graphed.master] + graphed.replicas, saved):
+            dst.copy_(src)
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(graphed.master, eager.master) and torch.equal(graphed.norms, eager.norms)
+        for a, b in zip(graphed.replicas, eager.replicas):
+            assert torch.equal(a, b)
+    L.lossy_device_status(graphed.ctx)
