@@ -93,7 +93,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 }
 
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
-constexpr uint32_t kTmaSmemFixed = 128 + kMaxStages * sizeof(StageHdr);
+constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * sizeof(StageHdr);
 
 // Launch policy of the bulk-copy pipeline, from sweeps on B200 over W = 2..64, p = 0.05..0.3
 // (bandwidths in profiles/): which of the four builds runs and whether its bulk copies carry an

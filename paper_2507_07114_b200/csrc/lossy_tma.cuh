@@ -2,8 +2,8 @@
 //
 // One CTA = CW compute warps + 1 producer warp + 1 store warp (see TmaShape for the two builds).
 // The bucket's full packets are cut into tiles of at most kTile contiguous elements inside one
-// packet (kTile = 128 * CW), so one set of delivery masks covers a tile. Per tile and per group of up to GS (4 or 8) workers
-// the producer arms an mbarrier and issues 1-D bulk copies global -> shared memory for the
+// packet (kTile = 128 * CW), so one set of delivery masks covers a tile. Per tile and per group of
+// up to GS (4 or 8) workers the producer arms an mbarrier and issues 1-D bulk copies global -> shared memory for the
 // DELIVERED workers' pieces only (dropped packets are never read) and, with the last group, for
 // theta / m / v. Compute warps sum the pieces in ascending worker order from shared memory,
 // divide by the received count, run the optimizer in place in shared memory and write the wire
@@ -31,8 +31,9 @@ template <int CW> struct TmaShape {
   static constexpr int kCtasPerSm = CW >= 16 ? 1 : 2;
 };
 constexpr int kStaleBatch = 4;                            // stale replica packets in flight per compute lane (8 measured slower)
-constexpr int kGroupMax = 8;                              // workers per pipeline stage: template GS = 4 or 8
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 4;                             // deeper pipelines measured no faster
+constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 x kMaxStages x 8 B) and the abort flag
+static_assert(3 * kMaxStages * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
 constexpr uint32_t kMaxPolls = 1u << 22;
 
 struct TmaGeom {
@@ -189,11 +190,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   constexpr int kTile = TmaShape<CW>::kTile;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
-  // layout: [full, done, empty barriers | abort flag] (128 B) | headers (kMaxStages x 64 B) | stages
+  // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) | stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
-  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + 96);
-  StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + 128);
-  unsigned char* stage0 = smem + 128 + kMaxStages * sizeof(StageHdr);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kTmaBarBytes - 4);
+  StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + kTmaBarBytes);
+  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr);
   const uint32_t S = G.stages;
   const uint32_t off_th = G.grad_slots * kTile * kGB;
   const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4, off_wire = off_v + kTile * 4;
@@ -355,11 +356,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint64_t stale = h.stale, e0 = h.e0;
         float wire[kEpl];
         if (active) {
-          if (cnt > 0) {
-            const float fc = (float)cnt;
-#pragma unroll
-            for (int x = 0; x < kEpl; ++x) acc[x] = __fdiv_rn(acc[x], fc);
-          }
+          divide_by_count<kEpl>(acc, cnt);
           if (P.ghat_prev) {
             // Algorithm 1: a dropped packet falls back to the saved aggregate, a surviving one is saved
             uint32_t pw[4];
