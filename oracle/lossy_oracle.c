@@ -131,6 +131,9 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
  *                   a transmission is lost iff its link is bad at step t. p_grad / p_param are unused.
  *   burst_in/out    [2][packets] uint64 (row 0 gradient links, row 1 broadcast links; bit i = link of
  *                   worker i is bad): state after step t-1 (read) and after step t (written)
+ *   reliable        optional [2][packets] uint64 (row 0 gradient links, row 1 broadcast links): bit i set =
+ *                   that transmission travels on a reliable channel and is never lost (the hybrid
+ *                   reliable/unreliable transport of the paper's Future Directions)
  *   recv_force      optional [packets] uint64: use these delivery bits (bit i = s_i)
  *                   instead of the hash — the hook the exhaustive-pattern test uses
  *                   (Algorithm 1 mode: bit 0 = the packet's aggregate survives)
@@ -144,7 +147,7 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
 int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_slab,
                const void* const* grads, REAL* master, REAL* m, REAL* v, void* const* replicas,
                REAL* ghat_prev, const double* burst, const uint64_t* burst_in, uint64_t* burst_out,
-               const uint64_t* recv_force, const uint64_t* stale_force,
+               const uint64_t* reliable, const uint64_t* recv_force, const uint64_t* stale_force,
                REAL* ghat, uint8_t* count, uint64_t* recv_bits, uint64_t* stale_bits,
                uint32_t* const* age, double* sumsq) {
   if (!c || c->W == 0 || c->W > 64 || c->packet_elems == 0) return 1;
@@ -209,6 +212,12 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
         }
         if (s) recv |= 1ULL << i;
       }
+    if (reliable && !recv_force) {
+      const uint64_t all = W == 64 ? ~0ULL : ((1ULL << W) - 1ULL);
+      /* Algorithm 1 mode has one transmission per packet: bit 0 makes it reliable */
+      if (ghat_prev) { if (reliable[kl] & 1ULL) recv = all; }
+      else recv |= reliable[kl] & all;
+    }
     uint32_t cnt = 0;
     for (uint32_t i = 0; i < W; ++i) cnt += (uint32_t)((recv >> i) & 1ULL);
     if (count) count[kl] = (uint8_t)cnt;
@@ -229,6 +238,7 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
       for (uint32_t i = 0; i < W; ++i)
         if (i != j && NAME(hash_u32)(c->seed, step, j, i, kg) < Tp) stale |= 1ULL << i;
     if (burst) { burst_out[kl] = gbad; burst_out[packets + kl] = pbad; }
+    if (reliable && !stale_force) stale &= ~reliable[packets + kl];
     if (stale_bits) stale_bits[kl] = stale;
 
     for (uint64_t e = e0; e < e1; ++e) {
@@ -350,6 +360,26 @@ int NAME(pairwise_sumsq)(const oracle_config* c, uint64_t n_slab, const void* co
         double d = ri - rk;
         d2[(size_t)i * W + k] += d * d;
       }
+    }
+  return 0;
+}
+
+/*
+ * Per (worker, packet) squared norm of the gradient pieces, the input of an importance rule
+ * ("large-norm gradients ... would traverse a reliable channel"): out[i * packets + k] in double.
+ */
+int NAME(packet_sqnorms)(const oracle_config* c, uint64_t n_slab, const void* const* grads, double* out) {
+  if (!c || !grads || !out) return 1;
+  const uint64_t P = c->packet_elems, packets = (n_slab + P - 1) / P;
+  for (uint32_t i = 0; i < c->W; ++i)
+    for (uint64_t k = 0; k < packets; ++k) {
+      double s = 0.0;
+      const uint64_t e1 = (k + 1) * P < n_slab ? (k + 1) * P : n_slab;
+      for (uint64_t e = k * P; e < e1; ++e) {
+        double g = (double)load_grad(grads[i], c->grad_dtype, e);
+        s += g * g;
+      }
+      out[(size_t)i * packets + k] = s;
     }
   return 0;
 }

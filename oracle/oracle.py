@@ -78,10 +78,13 @@ def _lib(f64: bool):
         o.argtypes = [C.POINTER(OracleConfig), C.c_uint64]
         s = getattr(lib, pre + "step")
         s.restype = C.c_int
-        s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 17
+        s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 18
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
         ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
+        sq = getattr(lib, pre + "packet_sqnorms")
+        sq.restype = C.c_int
+        sq.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p]
         pw = getattr(lib, pre + "pairwise_sumsq")
         pw.restype = C.c_int
         pw.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p]
@@ -167,7 +170,19 @@ class Oracle:
     def set_lr(self, lr: float) -> None:
         self.cfg.lr = lr
 
-    def step(self, t, grads, *, recv_force=None, stale_force=None, want_ghat=True):
+    def packet_sqnorms(self, grads):
+        """[W][packets] squared norms of the gradient pieces, in double."""
+        gd = np.uint16 if self.grad_dtype == BF16 else np.float32
+        grads = [np.ascontiguousarray(g, dtype=gd) for g in grads]
+        out = np.zeros((self.W, self.packets), np.float64)
+        gt = _ptr_table(grads)
+        rc = getattr(self.lib, self.pre + "packet_sqnorms")(C.byref(self.cfg), self.n_slab, C.cast(gt, C.c_void_p),
+                                                            _ptr(out))
+        if rc != 0:
+            raise ValueError("oracle_packet_sqnorms rejected its arguments")
+        return out
+
+    def step(self, t, grads, *, recv_force=None, stale_force=None, want_ghat=True, reliable=None):
         """Advance one iteration; returns a dict of ghat, count, recv_bits, stale_bits, sumsq, norms."""
         gd = np.uint16 if self.grad_dtype == BF16 else np.float32
         grads = [np.ascontiguousarray(g, dtype=gd) for g in grads]
@@ -184,10 +199,13 @@ class Oracle:
         if stale_force is not None:
             stale_force = np.ascontiguousarray(stale_force, dtype=np.uint64)
         burst_out = np.zeros_like(self.burst_state) if self.burst is not None else None
+        if reliable is not None:        # [2][packets]: reliable gradient links, reliable broadcast links
+            reliable = np.ascontiguousarray(reliable, dtype=np.uint64)
+            assert reliable.shape == (2, self.packets)
         rc = getattr(self.lib, self.pre + "step")(
             C.byref(self.cfg), t, self.k0, self.n_slab, C.cast(gt, C.c_void_p), _ptr(self.master),
             _ptr(self.m), _ptr(self.v), C.cast(rt, C.c_void_p), _ptr(self.ghat_prev), _ptr(self.burst),
-            _ptr(self.burst_state), _ptr(burst_out), _ptr(recv_force), _ptr(stale_force),
+            _ptr(self.burst_state), _ptr(burst_out), _ptr(reliable), _ptr(recv_force), _ptr(stale_force),
             _ptr(ghat), _ptr(count), _ptr(recv), _ptr(stale),
             C.cast(at, C.c_void_p) if at is not None else None, _ptr(sumsq))
         if rc != 0:
