@@ -128,6 +128,30 @@ int lossy_set_lr(lossy_ctx* ctx, float lr);
 int lossy_set_bursty(lossy_ctx* ctx, double p_enter_bad, double p_leave_bad, uint64_t* state);
 
 /*
+ * lossy_set_reliable — hybrid reliable/unreliable transport, the first of the
+ * paper's Future Directions ("large-norm gradients ... would traverse a reliable
+ * channel, while the long tail of small-magnitude updates would continue over a
+ * best-effort stream"): transmissions whose bit is set are never lost.
+ *   reliable  device, caller-owned, 2*K uint64: row 0 gradient links (bit i of entry
+ *             k = worker i's piece of packet k), row 1 broadcast links (bit i = the
+ *             broadcast of packet k to replica i). Read at every later call; the
+ *             caller may rewrite it between steps. NULL = everything best-effort.
+ * In Algorithm 1 mode bit 0 of row 0 makes the packet's single transmission reliable.
+ * The estimator is then no longer the unbiased one of the paper (reliable pieces are
+ * over-represented); the paper gives no correction and none is applied.
+ */
+int lossy_set_reliable(lossy_ctx* ctx, const uint64_t* reliable);
+
+/*
+ * lossy_packet_sqnorms — what an importance rule starts from: the squared L2 norm
+ * of every gradient piece, out[i*K + k] = sum over packet k of float(g_i[e])^2
+ * (fp32, fixed summation order).
+ *   grads  host array of W device pointers, each [n] of cfg.grad_dtype
+ *   out    [W*K] fp32 device, written
+ */
+int lossy_packet_sqnorms(lossy_ctx* ctx, const void* const* grads, float* out, void* stream);
+
+/*
  * lossy_aggregate — Section 3 step (2) and "Unbiased Gradient Aggregation":
  * for every packet k with owner j,
  *     s_i   = 1 iff hash(seed, step, src=i, dst=j, packet_base+k) >= T_grad

@@ -20,7 +20,7 @@ LOSSY_SGD, LOSSY_ADAM = 0, 1
 LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
 
 EXPORTS = [
-    "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_aggregate", "lossy_step", "lossy_broadcast",
+    "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_set_reliable", "lossy_packet_sqnorms", "lossy_aggregate", "lossy_step", "lossy_broadcast",
     "drift_norms", "drift_pairwise", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
 ]
@@ -64,6 +64,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_set_lr.argtypes = [vp, C.c_float]
     lib.lossy_set_bursty.restype = C.c_int
     lib.lossy_set_bursty.argtypes = [vp, C.c_double, C.c_double, vp]
+    lib.lossy_set_reliable.restype = C.c_int
+    lib.lossy_set_reliable.argtypes = [vp, vp]
+    lib.lossy_packet_sqnorms.restype = C.c_int
+    lib.lossy_packet_sqnorms.argtypes = [vp, vp, vp, vp]
     lib.lossy_aggregate.restype = C.c_int
     lib.lossy_aggregate.argtypes = [vp, u64, vp, vp, vp, vp, vp]
     lib.lossy_step.restype = C.c_int
@@ -157,6 +161,15 @@ def lossy_set_lr(ctx, lr):
 def lossy_set_bursty(ctx, p_enter_bad, p_leave_bad, state):
     """state: int64/uint64 device tensor of 4*K elements, zeroed before step 1; None = independent loss."""
     _check(ctx, load_library().lossy_set_bursty(ctx, p_enter_bad, p_leave_bad, _p(state)))
+
+
+def lossy_set_reliable(ctx, reliable):
+    """reliable: int64/uint64 device tensor of 2*K elements (row 0 gradient links, row 1 broadcast links) or None."""
+    _check(ctx, load_library().lossy_set_reliable(ctx, _p(reliable)))
+
+
+def lossy_packet_sqnorms(ctx, grads, out):
+    _check(ctx, load_library().lossy_packet_sqnorms(ctx, _table(grads), _p(out), _stream()))
 
 
 def lossy_aggregate(ctx, step, grads, ghat, count=None, recv_bits=None):

@@ -26,6 +26,7 @@ struct lossy_ctx {
   uint32_t* status;      // device status word: 0 = fine, 1 = a bounded wait in a kernel gave up
   uint32_t* ticket;      // device counter of finished blocks (last-block drift finalisation), zero between calls
   bool plan_only;        // launch helpers only report their grid size
+  const uint64_t* reliable;  // caller-owned device array [2][K] of reliable-link bits, or NULL
   uint64_t* burst_state; // bursty loss: caller-owned device array [2 buffers][2 rows][K], or NULL
   uint32_t Tenter, Tstay;
   int smem_optin;        // largest dynamic shared memory a block may opt in to
@@ -82,6 +83,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   P.eps = c.eps;
   P.partials = ctx->partials;
   P.K = (uint32_t)ctx->K;
+  P.reliable = ctx->reliable;
   if (ctx->burst_state) {
     // the states after step t-1 live in buffer (t-1)&1, those after step t go to buffer t&1
     const size_t buf = 2 * (size_t)ctx->K;
@@ -327,6 +329,39 @@ int lossy_set_bursty(lossy_ctx* ctx, double p_enter_bad, double p_leave_bad, uin
   ctx->burst_state = state;
   ctx->Tenter = threshold_of(p_enter_bad);
   ctx->Tstay = p_leave_bad >= 1.0 ? 0u : threshold_of(1.0 - p_leave_bad);
+  return LOSSY_OK;
+}
+
+int lossy_set_reliable(lossy_ctx* ctx, const uint64_t* reliable) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (reinterpret_cast<uintptr_t>(reliable) & 7u) return fail(ctx, LOSSY_EINVAL, "reliable: misaligned");
+  if (ctx->K >= (1ull << 32)) return fail(ctx, LOSSY_EINVAL, "too many packets");
+  ctx->reliable = reliable;
+  return LOSSY_OK;
+}
+
+int lossy_packet_sqnorms(lossy_ctx* ctx, const void* const* grads, float* out, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (!out) return fail(ctx, LOSSY_EINVAL, "out: NULL");
+  if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  SqnormArgs A;
+  memset(&A, 0, sizeof A);
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) A.grads[i] = grads[i];
+  A.out = out;
+  A.n = ctx->cfg.n;
+  A.W = ctx->cfg.W;
+  A.P = ctx->cfg.packet_elems;
+  A.K = (uint32_t)ctx->K;
+  uint64_t blocks = ((uint64_t)A.W * A.K + 7) / 8;
+  const uint64_t cap = (uint64_t)ctx->num_sms * 8;
+  if (blocks > cap) blocks = cap;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (ctx->cfg.grad_dtype == LOSSY_BF16) packet_sqnorms_kernel<BF16><<<(uint32_t)blocks, 256, 0, s>>>(A);
+  else packet_sqnorms_kernel<F32><<<(uint32_t)blocks, 256, 0, s>>>(A);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "packet norm launch", e);
+  ctx->launches++;
   return LOSSY_OK;
 }
 

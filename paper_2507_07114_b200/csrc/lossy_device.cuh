@@ -45,6 +45,7 @@ struct Params {
   uint32_t total_rows;    // partial rows (= blocks) of the whole call
   float* norms;           // [W] or NULL
   double* sumsq;          // [W], added to, or NULL
+  const uint64_t* reliable;  // [2][K] (row 0 gradient links, row 1 broadcast links): set bits are never lost; or NULL
   const uint64_t* burst_in;  // bursty loss: link states after the previous step, [2][K] (row 0 gradient links, row 1 broadcast links)
   uint64_t* burst_out;       // link states after this step, same layout (a different buffer)
   uint64_t n;

@@ -108,6 +108,12 @@ __device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32
     }
     recv = ((uint64_t)hi << 32) | lo;
     gbad = alg1 ? (uint64_t)(blo & 1u) : (((uint64_t)bhi << 32) | blo);
+    if (P.reliable) {   // transmissions on the reliable channel always arrive
+      const uint64_t all = W == 64 ? ~0ull : ((1ull << W) - 1ull);
+      const uint64_t rel = P.reliable[k];
+      if (alg1) { if (rel & 1ull) recv = all; }
+      else recv |= rel & all;
+    }
   }
   if constexpr (PH & BCAST) {
     const uint64_t pin = bursty ? P.burst_in[(size_t)P.K + k] : 0ull;
@@ -123,6 +129,7 @@ __device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32
     }
     stale = ((uint64_t)hi << 32) | lo;
     pbad = stale;
+    if (P.reliable) stale &= ~P.reliable[(size_t)P.K + k];
   }
 }
 template <int PH>
@@ -358,6 +365,35 @@ static __global__ void drift_finalize_kernel(const double* __restrict__ partials
   if (threadIdx.x == 0) {
     if (sumsq) sumsq[i] += t;
     if (norms) norms[i] = (float)sqrt(t);
+  }
+}
+
+// Squared norm of every (worker, packet) gradient piece: out[i * K + k]. One warp per piece.
+struct SqnormArgs {
+  const void* grads[kMaxW];
+  float* out;
+  uint64_t n;
+  uint32_t W, P, K;
+};
+template <class GT>
+static __global__ void __launch_bounds__(256) packet_sqnorms_kernel(const __grid_constant__ SqnormArgs A) {
+  const int lane = threadIdx.x & 31;
+  const uint64_t warps = (uint64_t)gridDim.x * (blockDim.x >> 5);
+  const uint64_t tasks = (uint64_t)A.W * A.K;
+  for (uint64_t task = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); task < tasks; task += warps) {
+    const uint32_t i = (uint32_t)(task / A.K), k = (uint32_t)(task % A.K);
+    const uint64_t e0 = (uint64_t)k * A.P;
+    const uint64_t e1 = e0 + A.P < A.n ? e0 + A.P : A.n;
+    float s = 0.0f;
+    for (uint64_t e = e0 + (uint64_t)lane * 8; e < e1; e += 256) {
+      const int nvalid = e1 - e >= 8 ? 8 : (int)(e1 - e);
+      float f[8];
+      widen<GT>(load8_any<GT>(A.grads[i], e, nvalid), f);
+#pragma unroll
+      for (int x = 0; x < 8; ++x) s = __fadd_rn(s, x < nvalid ? __fmul_rn(f[x], f[x]) : 0.0f);
+    }
+    s = warp_sum(s);
+    if (lane == 0) A.out[(size_t)i * A.K + k] = s;
   }
 }
 
