@@ -44,6 +44,7 @@ def assert_rel(got, want, what, tol=REL_TOL):
     assert got.shape == want.shape, what
     if got.size == 0:
         return
+    got, want = got.ravel(), want.ravel()
     err = np.abs(got - want) / np.maximum(np.abs(want), TINY)
     bad = int(np.argmax(err))
     assert err[bad] <= tol, f"{what}: rel err {err[bad]:.3e} at {bad} (got {got[bad]!r}, want {want[bad]!r})"
