@@ -23,6 +23,8 @@
  *   - `step` is 1-based: it is the hash's step counter and Adam's t.
  *   - Return value: LOSSY_OK or an error code; nothing throws, nothing traps on
  *     the device. A bad argument is rejected before any launch.
+ *   - A context owns scratch that its calls share (partial sums, a block counter):
+ *     issue the calls of one context on one stream, or order them with events.
  *   - The bucket is cut into K = ceil(n / packet_elems) packets of
  *     `packet_elems` contiguous elements (the last may be short). Shard j, owned
  *     by worker j, is the contiguous packet range [j*pps, min(K,(j+1)*pps)) with
@@ -129,9 +131,9 @@ int lossy_set_bursty(lossy_ctx* ctx, double p_enter_bad, double p_leave_bad, uin
 
 /*
  * lossy_set_reliable — hybrid reliable/unreliable transport, the first of the
- * paper's Future Directions ("large-norm gradients ... would traverse a reliable
- * channel, while the long tail of small-magnitude updates would continue over a
- * best-effort stream"): transmissions whose bit is set are never lost.
+ * paper's Future Directions: traffic classed as important (there: gradients of
+ * large norm) goes over a reliable channel, the rest stays best-effort.
+ * Transmissions whose bit is set here are never lost.
  *   reliable  device, caller-owned, 2*K uint64: row 0 gradient links (bit i of entry
  *             k = worker i's piece of packet k), row 1 broadcast links (bit i = the
  *             broadcast of packet k to replica i). Read at every later call; the
@@ -278,9 +280,9 @@ int lossy_fused_step(lossy_ctx* ctx, uint64_t step, const void* const* grads,
  * fp32, divided by W), then ONE draw per packet,
  *     keep = hash(seed, step, src=owner, dst=owner, packet_base+k) >= T_grad,
  * decides: keep => ghat = mean and ghat_prev <- mean; drop => ghat = ghat_prev and
- * ghat_prev is left as it was (Algorithm 1: "drop gradient: g <- g_prev, else
- * g_prev <- g"). "Renormalise surviving shards" is read as the division of the
- * reduced sum by the worker count. Shard-granular loss, as the algorithm prints it,
+ * ghat_prev is left as it was (the two branches of Algorithm 1's gradient loop).
+ * The algorithm's renormalisation step is read as the division of the reduced
+ * sum by the worker count. Shard-granular loss, as the algorithm prints it,
  * is packet_elems = shard length. The parameter half (stale-retaining broadcast with
  * p_param) and everything else are those of lossy_aggregate / lossy_fused_step.
  *   ghat_prev  [n] fp32 device, caller-owned state, zero before the first step;

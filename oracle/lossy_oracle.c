@@ -366,7 +366,7 @@ int NAME(pairwise_sumsq)(const oracle_config* c, uint64_t n_slab, const void* co
 
 /*
  * Per (worker, packet) squared norm of the gradient pieces, the input of an importance rule
- * ("large-norm gradients ... would traverse a reliable channel"): out[i * packets + k] in double.
+ * (Future Directions: gradients of large norm are the traffic to send reliably): out[i * packets + k], double.
  */
 int NAME(packet_sqnorms)(const oracle_config* c, uint64_t n_slab, const void* const* grads, double* out) {
   if (!c || !grads || !out) return 1;
