@@ -98,7 +98,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * sizeof(StageHdr);
 
 // Launch policy of the bulk-copy pipeline, from sweeps on B200 over W = 2..64, p = 0.05..0.3
-// (bandwidths in profiles/): which of the four builds runs and whether its bulk copies carry an
+// (CUDA-event timings of bench.py with each build forced): which of the four builds runs and whether its bulk copies carry an
 // L2 evict-first hint (bit 0 loads, bit 1 stores).
 struct TmaPolicy {
   bool wide;      // 16 compute warps, one CTA per SM, 2048-element tiles (else 8 warps, two CTAs, 1024)
