@@ -1,6 +1,6 @@
 """Throughput and drift of the fused step over the benchmark configurations.
 
-    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,5,alg1] [--steps N]
+    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,5,alg1,unfused] [--steps N]
 
 Prints one line per point: algorithmic GB/s, fraction of the measured HBM copy peak, steps/s and the
 largest per-replica drift norm seen. Inputs are the seeded synthetic workloads; state stays in HBM.
@@ -101,6 +101,49 @@ def run_point(w, steps, warmup=3, grad_sets=2, alg1=False, graph=False):
             **({"steps_per_s_cuda_graph": graph_sps} if graph_sps else {})}
 
 
+def run_unfused(w, steps=20, warmup=3):
+    """Each unfused entry point on its own: time and algorithmic GB/s of aggregate, step, broadcast, drift."""
+    dev = torch.device("cuda")
+    gdt = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    rdt = torch.bfloat16 if w.replica_dtype == "bf16" else torch.float32
+    gb, rb = (2 if w.grad_dtype == "bf16" else 4), (2 if w.replica_dtype == "bf16" else 4)
+    adam = w.optimizer == "adam"
+    ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems, p_grad=w.p, p_param=w.p, seed=w.seed,
+                       grad_dtype=gdt, replica_dtype=rdt, optimizer=w.optimizer, lr=w.lr, beta1=w.beta1,
+                       beta2=w.beta2, eps=w.eps)
+    master = workload.theta0_slab(w, 0, w.n, dev)
+    m = torch.zeros_like(master) if adam else None
+    v = torch.zeros_like(master) if adam else None
+    reps = [master.to(rdt) for _ in range(w.W)]
+    grads = [workload.grad_slab(w, 1, i, 0, w.n, dev) for i in range(w.W)]
+    ghat = torch.zeros_like(master)
+    count = torch.zeros(w.K, dtype=torch.uint8, device=dev)
+    norms = torch.zeros(w.W, device=dev)
+    n, W, p = w.n, w.W, w.p
+    calls = {
+        "lossy_aggregate": (lambda t: L.lossy_aggregate(ctx, t, grads, ghat, count), (1 - p) * W * n * gb + 4 * n),
+        "lossy_step": (lambda t: L.lossy_step(ctx, t, ghat, count, master, m, v), (28 if adam else 12) * n),
+        "lossy_broadcast": (lambda t: L.lossy_broadcast(ctx, t, master, reps), 4 * n + ((W - 1) * (1 - p) + 1) * n * rb),
+        "drift_norms": (lambda t: L.drift_norms(ctx, master, reps, norms), 4 * n + W * n * rb),
+    }
+    out = []
+    for name, (fn, nbytes) in calls.items():
+        for t in range(1, warmup + 1):
+            fn(t)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(warmup + 1, warmup + steps + 1):
+            fn(t)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        out.append({"workload": w.name, "call": name, "ms": ms, "GBps": nbytes / (ms * 1e-3) / 1e9,
+                    "frac_of_measured_peak": nbytes / (ms * 1e-3) / 1e9 / _peak()})
+    L.lossy_destroy(ctx)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,5")
@@ -123,6 +166,9 @@ def main():
     for w in points:
         r = run_point(w, args.steps or w.steps, grad_sets=1 if w.W >= 64 else 2, graph=w.n <= (1 << 22))
         print(json.dumps(r), flush=True)
+    if "unfused" in want:
+        for r in run_unfused(cfg["cfg2_w8_layer_adam"]):
+            print(json.dumps(r), flush=True)
     if "alg1" in want:
         # Algorithm 1 mode on the config-2 bucket: packet-granular and shard-granular (P = n / W) drops
         base = cfg["cfg2_w8_layer_adam"]
