@@ -300,12 +300,15 @@ int lossy_fused_step_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grad
 
 /*
  * lossy_fused_step_host — the same step for a caller whose gradients live in
- * HOST memory (pinned memory for full copy speed): copies worker i's gradient
- * from host_grads[i] into dev_grads[i] on `stream`, runs lossy_fused_step, and
- * copies the W norms to `host_norms`. It returns after the stream has been
+ * HOST memory, with the W norms delivered to host memory.
+ * Pinned (page-locked, device-mapped) buffers are read by the kernel directly over
+ * PCIe: there is no staging copy, and the packets the network dropped are never
+ * transferred at all. If any buffer is pageable, every worker's gradient is first
+ * copied into dev_grads[i] on `stream`. The call returns after the stream has been
  * synchronised (through lossy_device_status), so `host_norms` is valid on return.
- *   host_grads  host array of W HOST pointers, each [n] of cfg.grad_dtype
- *   dev_grads   host array of W DEVICE staging pointers, each [n], caller-owned
+ *   host_grads  host array of W HOST pointers, each [n] of cfg.grad_dtype, 16-byte aligned
+ *   dev_grads   host array of W DEVICE staging pointers, each [n], caller-owned; only
+ *               used (and only then required to be non-NULL) for pageable host memory
  *   dev_norms   [W] fp32 device; host_norms [W] fp32 host
  */
 int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host_grads,

@@ -227,8 +227,10 @@ def lossy_fused_step_alg1(ctx, step, grads, ghat_prev, master, m, v, replicas, g
 
 
 def lossy_fused_step_host(ctx, step, host_grads, dev_grads, master, m, v, replicas, dev_norms, host_norms):
-    """host_grads: W pinned CPU tensors; host_norms: a CPU fp32 tensor of W elements (valid on return)."""
-    _check(ctx, load_library().lossy_fused_step_host(ctx, step, _table(host_grads), _table(dev_grads), _p(master),
+    """host_grads: W CPU tensors (pinned: read in place over PCIe; pageable: staged through dev_grads, which
+    may be None otherwise); host_norms: a CPU fp32 tensor of W elements (valid on return)."""
+    _check(ctx, load_library().lossy_fused_step_host(ctx, step, _table(host_grads),
+                                                     None if dev_grads is None else _table(dev_grads), _p(master),
                                                      _p(m), _p(v), _table(replicas), _p(dev_norms), _p(host_norms),
                                                      _stream()))
 

@@ -627,17 +627,33 @@ int lossy_fused_step_host(lossy_ctx* ctx, uint64_t step, const void* const* host
                           float* master, float* m, float* v, void* const* replicas, float* dev_norms,
                           float* host_norms, void* stream) {
   if (!ctx) return LOSSY_EINVAL;
-  if (!host_grads || !dev_grads || !dev_norms || !host_norms) return fail(ctx, LOSSY_EINVAL, "NULL argument");
+  if (!host_grads || !dev_norms || !host_norms) return fail(ctx, LOSSY_EINVAL, "NULL argument");
   cudaStream_t s = (cudaStream_t)stream;
   const size_t gbytes = (size_t)ctx->cfg.n * (ctx->cfg.grad_dtype == LOSSY_BF16 ? 2 : 4);
+  // Zero-copy: when every host buffer is pinned and mapped into the device's address space, the kernel
+  // reads the gradients over PCIe itself, so packets that the network dropped are never transferred at all
+  // and no staging copy is made. Otherwise (pageable memory) each buffer is staged with cudaMemcpyAsync.
+  const void* mapped[LOSSY_MAX_WORKERS];
+  bool zero_copy = true;
   for (uint32_t i = 0; i < ctx->cfg.W; ++i) {
-    if (!host_grads[i] || !dev_grads[i]) return fail(ctx, LOSSY_EINVAL, "NULL gradient pointer");
-    if (gbytes) {
-      cudaError_t e = cudaMemcpyAsync(dev_grads[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, s);
-      if (e != cudaSuccess) return fail_cuda(ctx, "gradient upload", e);
-    }
+    if (!host_grads[i]) return fail(ctx, LOSSY_EINVAL, "NULL gradient pointer");
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_grads[i]) != cudaSuccess) { cudaGetLastError(); zero_copy = false; continue; }
+    if (attr.type != cudaMemoryTypeHost || !attr.devicePointer || !aligned16(attr.devicePointer)) zero_copy = false;
+    mapped[i] = attr.devicePointer;
   }
-  if (int rc = lossy_fused_step(ctx, step, dev_grads, master, m, v, replicas, nullptr, nullptr, nullptr, nullptr,
+  const void* const* step_grads = mapped;
+  if (!zero_copy) {
+    for (uint32_t i = 0; i < ctx->cfg.W; ++i) {
+      if (!dev_grads || !dev_grads[i]) return fail(ctx, LOSSY_EINVAL, "pageable host gradients need staging buffers");
+      if (gbytes) {
+        cudaError_t e = cudaMemcpyAsync(dev_grads[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return fail_cuda(ctx, "gradient upload", e);
+      }
+    }
+    step_grads = dev_grads;
+  }
+  if (int rc = lossy_fused_step(ctx, step, step_grads, master, m, v, replicas, nullptr, nullptr, nullptr, nullptr,
                                 dev_norms, nullptr, stream))
     return rc;
   cudaError_t e = cudaMemcpyAsync(host_norms, dev_norms, ctx->cfg.W * sizeof(float), cudaMemcpyDeviceToHost, s);

@@ -267,3 +267,28 @@ def test_ten_steps_captured_in_a_cuda_graph_replay_bit_identically():
         for a, b in zip(graphed.replicas, eager.replicas):
             assert torch.equal(a, b)
     L.lossy_device_status(graphed.ctx)
+
+
+def test_host_gradient_entry_point_zero_copy_and_staged_match_the_device_path():
+    """lossy_fused_step_host: pinned host gradients are read in place by the kernel, pageable ones are staged;
+    both leave exactly the state of lossy_fused_step on device-resident gradients."""
+    w = workload.scaled(CFG["cfg2_w8_layer_adam"], 2048 * 41 + 1003)
+    ref, pinned, paged = GpuRun(w), GpuRun(w), GpuRun(w)
+    staging = [torch.empty(w.n, dtype=torch.bfloat16, device="cuda") for _ in range(w.W)]
+    host_norms = torch.zeros(w.W)
+    for t in range(1, 5):
+        gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]
+        ref.step_fused(t, [g.cuda() for g in gs], outputs=False)
+        L.lossy_fused_step_host(pinned.ctx, t, [g.pin_memory() for g in gs], None, pinned.master, pinned.m, pinned.v,
+                                pinned.replicas, pinned.norms, host_norms)
+        assert torch.equal(host_norms, ref.norms.cpu())
+        L.lossy_fused_step_host(paged.ctx, t, gs, staging, paged.master, paged.m, paged.v, paged.replicas,
+                                paged.norms, host_norms)
+        assert torch.equal(host_norms, ref.norms.cpu())
+        for run in (pinned, paged):
+            assert torch.equal(run.master, ref.master) and torch.equal(run.v, ref.v)
+            for a, b in zip(run.replicas, ref.replicas):
+                assert torch.equal(a, b)
+    with pytest.raises(L.LossyError):                      # pageable memory without staging buffers
+        L.lossy_fused_step_host(paged.ctx, 5, gs, None, paged.master, paged.m, paged.v, paged.replicas, paged.norms,
+                                host_norms)
