@@ -103,6 +103,7 @@ constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * sizeof(StageHdr);
 struct TmaPolicy {
   bool wide;      // 16 compute warps, one CTA per SM, 2048-element tiles (else 8 warps, two CTAs, 1024)
   int group;      // workers per pipeline stage: 4 or 8
+  bool early_stale;  // request the first stale replica copies before the tile's arithmetic (stages of 8 only)
   uint32_t hints;
 };
 TmaPolicy tma_policy(const lossy_config& c) {
@@ -115,6 +116,9 @@ TmaPolicy tma_policy(const lossy_config& c) {
   t.group = c.W <= 4 ? 4 : (c.W <= 8 && pm < 0.175 ? 4 : 8);
   // hints: +3-4 % on the twin build at W = 64 or at high loss, neutral to -2 % elsewhere
   t.hints = t.wide ? (pm >= 0.28 ? 3u : 0u) : ((c.W > 32 || pm >= 0.2) ? 3u : 0u);
+  // early stale requests pay from about two stale replicas per tile at high loss: +8-10 % at W >= 16,
+  // p = 0.3; at p = 0.1 they lose 1-2 % even with six stale replicas per tile (W = 64)
+  t.early_stale = t.group == 8 && (c.W - 1) * c.p_param >= 2.0 && c.p_param >= 0.15;
   return t;
 }
 
@@ -154,9 +158,9 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   return true;
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE>
 int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS>;
+  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS, PRE>;
   constexpr int kThreadsTma = TmaShape<CW>::kThreads;
   const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
   // launch bounds and the shared-memory budget guarantee kCtasPerSm resident CTAs per SM
@@ -178,23 +182,24 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   return LOSSY_OK;
 }
 
-template <bool DRIFTK, int CW, int GS>
+template <bool DRIFTK, int CW, int GS, int PRE>
 int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
   const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
   const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
   const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
-  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
-  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
-  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
-  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS>(ctx, P, G, s, blocks);
+  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
+  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
 }
 
-template <int CW, int GS>
+template <int CW, int GS, int PRE = 0>
 int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
   TmaGeom G;
   if (!tma_geometry<CW, GS>(ctx, G)) return LOSSY_OK;
   *used = true;
-  return drift ? dispatch_tma<true, CW, GS>(ctx, P, G, s, blocks) : dispatch_tma<false, CW, GS>(ctx, P, G, s, blocks);
+  // without drift norms nothing reads the stale copies: the plain build serves
+  return drift ? dispatch_tma<true, CW, GS, PRE>(ctx, P, G, s, blocks) : dispatch_tma<false, CW, GS, 0>(ctx, P, G, s, blocks);
 }
 
 // Run the build the policy picks; *used stays false when no bulk-copy launch fits (packets shorter
@@ -204,10 +209,14 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
   const TmaPolicy t = tma_policy(ctx->cfg);
   if (t.wide) {
-    int rc = t.group == 4 ? try_tma<16, 4>(ctx, P, drift, s, blocks, used) : try_tma<16, 8>(ctx, P, drift, s, blocks, used);
+    int rc = t.group == 4 ? try_tma<16, 4>(ctx, P, drift, s, blocks, used)
+             : t.early_stale ? try_tma<16, 8, 16>(ctx, P, drift, s, blocks, used)
+                             : try_tma<16, 8>(ctx, P, drift, s, blocks, used);
     if (rc || *used) return rc;
   }
-  return t.group == 4 ? try_tma<8, 4>(ctx, P, drift, s, blocks, used) : try_tma<8, 8>(ctx, P, drift, s, blocks, used);
+  return t.group == 4 ? try_tma<8, 4>(ctx, P, drift, s, blocks, used)
+         : t.early_stale ? try_tma<8, 8, 16>(ctx, P, drift, s, blocks, used)
+                         : try_tma<8, 8>(ctx, P, drift, s, blocks, used);
 }
 
 template <int PH, class GT, class RT, int OPT>
