@@ -162,7 +162,8 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
     uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
     packet_masks<PH>(P, k, j, lane, recv, stale, gbad, pbad);
     // Pull the NEXT chunk of this warp toward L2 while this one is processed. Worth its
-    // instructions only when few workers feed a chunk (measured: +3..13 % for W <= 8, a loss above).
+    // instructions only in the fused kernel when few workers feed a chunk (measured: +3..13 % for W <= 8,
+    // a loss above, and a loss in the single-phase kernels).
     if (P.prefetch_next) {
       const uint32_t qn = q + warps_in_grid;
       if (qn < P.num_chunks) {
