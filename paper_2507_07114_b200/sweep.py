@@ -1,6 +1,6 @@
 """Throughput and drift of the fused step over the benchmark configurations.
 
-    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,5,alg1,unfused] [--steps N]
+    python -m paper_2507_07114_b200.sweep [--configs 1,2,3,4,5,alg1,unfused] [--steps N]
 
 Prints one line per point: algorithmic GB/s, fraction of the measured HBM copy peak, steps/s and the
 largest per-replica drift norm seen. Inputs are the seeded synthetic workloads; state stays in HBM.
@@ -144,6 +144,59 @@ def run_unfused(w, steps=20, warmup=3):
     return out
 
 
+def run_model_streamed(base, layers, steps, warmup=2):
+    """Configuration 4's mechanism at (nearly) full scale: a model streamed bucket by bucket. One context per
+    bucket with its own shard map and a running global packet id; one gradient buffer is reused for every bucket
+    (the masks still differ: they hash the global packet id). Model-level drift = sqrt of the summed squares."""
+    dev = torch.device("cuda")
+    emb = 32000 * 4096
+    sizes = [workload.LAYER_ELEMS] * layers + [emb, emb]
+    ctxs, state, pb = [], [], 0
+    for b, n in enumerate(sizes):
+        w = workload.scaled(base, n, packet_base=pb, seed=base.seed + b)
+        ctx = L.lossy_init(W=w.W, n=n, packet_elems=w.packet_elems, p_grad=w.p, p_param=w.p, seed=w.seed,
+                           grad_dtype=torch.bfloat16, replica_dtype=torch.bfloat16, optimizer="adam", lr=w.lr,
+                           beta1=w.beta1, beta2=w.beta2, eps=w.eps, packet_base=pb)
+        master = workload.theta0_slab(w, 0, n, dev)
+        state.append((master, torch.zeros_like(master), torch.zeros_like(master),
+                      [master.to(torch.bfloat16) for _ in range(w.W)]))
+        ctxs.append((ctx, w))
+        pb += w.K
+    big = workload.scaled(base, workload.LAYER_ELEMS)
+    grads = [workload.grad_slab(big, 1, i, 0, big.n, dev) for i in range(base.W)]
+    sumsq = torch.zeros(base.W, dtype=torch.float64, device=dev)
+    worst = torch.zeros(base.W, dtype=torch.float64, device=dev)
+    total_bytes = sum(algorithmic_bytes(w) for _, w in ctxs)
+
+    def model_step(t):
+        sumsq.zero_()
+        for (ctx, w), (master, m, v, reps) in zip(ctxs, state):
+            L.lossy_fused_step(ctx, t, [g[:w.n] for g in grads], master, m, v, reps, sumsq=sumsq)
+        torch.maximum(worst, sumsq, out=worst)
+
+    t = 0
+    for _ in range(warmup):
+        t += 1
+        model_step(t)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        t += 1
+        model_step(t)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    for ctx, _ in ctxs:
+        L.lossy_device_status(ctx)
+        L.lossy_destroy(ctx)
+    gbs = total_bytes / (ms * 1e-3) / 1e9
+    return {"workload": f"cfg4_cut_{layers}_layers_plus_embedding_and_head", "W": base.W, "P": base.packet_elems,
+            "p": base.p, "buckets": len(sizes), "elements": sum(sizes), "resident_GB": round(sum(sizes) * 28 / 1e9, 1),
+            "ms_per_step": ms, "GBps": gbs, "frac_of_measured_peak": gbs / _peak(), "steps_per_s": 1e3 / ms,
+            "max_drift_norm": float(worst.max().sqrt())}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,5")
@@ -166,6 +219,9 @@ def main():
     for w in points:
         r = run_point(w, args.steps or w.steps, grad_sets=1 if w.W >= 64 else 2, graph=w.n <= (1 << 22))
         print(json.dumps(r), flush=True)
+    if "4" in want:
+        # the full model (32 layers) needs 189 GB resident and does not fit one GPU: 24 layers + embedding + head
+        print(json.dumps(run_model_streamed(cfg["cfg4_w8_full_model"], 24, args.steps or 20)), flush=True)
     if "unfused" in want:
         for r in run_unfused(cfg["cfg2_w8_layer_adam"]):
             print(json.dumps(r), flush=True)
