@@ -94,7 +94,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 }
 
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
-constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * sizeof(StageHdr);
+constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale));
 
 // Launch policy of the bulk-copy pipeline, from sweeps on B200 over W = 2..64, p = 0.05..0.3
 // (CUDA-event timings of bench.py with each build forced): which of the four builds runs and whether its bulk copies carry an
@@ -131,14 +131,24 @@ uint32_t tma_smem_budget(const lossy_ctx* ctx) {
   return budget;
 }
 
-template <int CW, int GS>
+template <int CW, int GS, bool PACKED>
 bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   constexpr uint32_t kGroup = GS;
   constexpr uint32_t kTile = TmaShape<CW>::kTile;
   const lossy_config& c = ctx->cfg;
-  if (c.packet_elems < kTile) return false;
   const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
-  if (kfull == 0) return false;
+  if (kfull == 0 || kfull >= (1ull << 31)) return false;
+  G.packets_per_tile = 1;
+  G.full_packets = (uint32_t)kfull;
+  if (PACKED) {
+    // small packets: a tile packs 2, 4 or 8 whole packets; a compute warp's 128 elements stay inside one
+    if (c.packet_elems >= kTile || kTile % c.packet_elems != 0 || c.packet_elems % 128 != 0 ||
+        kTile / c.packet_elems > (uint32_t)kMaxSub)
+      return false;
+    G.packets_per_tile = kTile / c.packet_elems;
+  } else if (c.packet_elems < kTile) {
+    return false;
+  }
   const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
   G.grad_slots = c.W < (uint32_t)kGroup ? c.W : (uint32_t)kGroup;
   G.groups = (c.W + kGroup - 1) / kGroup;
@@ -148,8 +158,8 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
   G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
   if (G.stages > (uint32_t)kMaxStages) G.stages = kMaxStages;
-  G.tiles_per_packet = (c.packet_elems + kTile - 1) / kTile;
-  const uint64_t tiles = kfull * G.tiles_per_packet;
+  G.tiles_per_packet = PACKED ? 1u : (c.packet_elems + kTile - 1) / kTile;
+  const uint64_t tiles = PACKED ? (kfull + G.packets_per_tile - 1) / G.packets_per_tile : kfull * G.tiles_per_packet;
   if (tiles >= (1ull << 31)) return false;
   G.num_tiles = (uint32_t)tiles;
   G.status = ctx->status;
@@ -157,9 +167,9 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   return true;
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED>
 int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS, PRE>;
+  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS, PRE, PACKED>;
   constexpr int kThreadsTma = TmaShape<CW>::kThreads;
   const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
   // launch bounds and the shared-memory budget guarantee kCtasPerSm resident CTAs per SM
@@ -181,24 +191,25 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   return LOSSY_OK;
 }
 
-template <bool DRIFTK, int CW, int GS, int PRE>
+template <bool DRIFTK, int CW, int GS, int PRE, bool PACKED>
 int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
   const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
   const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
   const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
-  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
-  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
-  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
-  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS, PRE>(ctx, P, G, s, blocks);
+  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
+  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
 }
 
-template <int CW, int GS, int PRE = 0>
+template <int CW, int GS, int PRE = 0, bool PACKED = false>
 int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
   TmaGeom G;
-  if (!tma_geometry<CW, GS>(ctx, G)) return LOSSY_OK;
+  if (!tma_geometry<CW, GS, PACKED>(ctx, G)) return LOSSY_OK;
   *used = true;
   // without drift norms nothing reads the stale copies: the plain build serves
-  return drift ? dispatch_tma<true, CW, GS, PRE>(ctx, P, G, s, blocks) : dispatch_tma<false, CW, GS, 0>(ctx, P, G, s, blocks);
+  return drift ? dispatch_tma<true, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks)
+               : dispatch_tma<false, CW, GS, 0, PACKED>(ctx, P, G, s, blocks);
 }
 
 // Run the build the policy picks; *used stays false when no bulk-copy launch fits (packets shorter
@@ -207,6 +218,22 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   *used = false;
   if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
   const TmaPolicy t = tma_policy(ctx->cfg);
+  if (ctx->cfg.packet_elems < (uint32_t)TmaShape<8>::kTile) {
+    // Packets shorter than a tile: the PACKED builds, where they beat the register kernel. They fetch the
+    // dropped sub-packets too, so they win at low loss with a moderate worker count (+8..15 % at W = 8-16,
+    // P = 256-512, p <= 0.1) and lose at p >= 0.2 or W >= 32; below 256 elements the register kernel's
+    // 256-element chunks are mostly idle lanes and the PACKED build always wins.
+    const lossy_config& c = ctx->cfg;
+    const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
+    if (c.packet_elems < 256 || (pm <= 0.15 && c.W >= 4 && c.W <= 24)) {
+      if (c.W <= 16) {
+        int rc = try_tma<16, 8, 0, true>(ctx, P, drift, s, blocks, used);
+        if (rc || *used) return rc;
+      }
+      int rc = try_tma<8, 8, 0, true>(ctx, P, drift, s, blocks, used);
+      if (rc || *used) return rc;
+    }
+  }
   if (t.wide) {
     int rc = t.group == 4 ? try_tma<16, 4>(ctx, P, drift, s, blocks, used)
              : t.early_stale ? try_tma<16, 8, 16>(ctx, P, drift, s, blocks, used)

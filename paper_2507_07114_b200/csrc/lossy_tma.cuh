@@ -44,8 +44,19 @@ struct TmaGeom {
   uint32_t groups;            // ceil(W / GS)
   uint32_t grad_slots;        // min(W, GS)
   uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores
+  uint32_t packets_per_tile;  // PACKED build: whole small packets per tile (2, 4 or 8), else 1
+  uint32_t full_packets;      // PACKED build: complete packets of the bucket
   uint32_t* status;           // device status word (0 = fine)
 };
+
+// PACKED build, for packets shorter than a tile: a tile holds up to kMaxSub whole packets. The producer
+// fetches every worker's piece of the tile in ONE bulk copy each (bulk copies under ~2 KB run far below the
+// memory rate, and a single warp cannot evaluate eight packets' masks per tile fast enough); the masks are
+// evaluated by the compute warps instead, each for the one packet its 128 elements lie in, so dropped
+// sub-packets are fetched but never used. The store warp writes each replica the runs of consecutive
+// sub-packets whose broadcast it received.
+constexpr int kMaxSub = 8;
+struct __align__(16) PackedStale { uint64_t stale[kMaxSub]; };
 
 struct __align__(16) StageHdr {
   uint64_t recv, stale, e0;
@@ -186,7 +197,7 @@ __device__ __forceinline__ void pack_bf16_lane(const float (&f)[kEpl], uint32_t 
 // arithmetic) so that its latency is hidden; 0 = every stale copy is fetched in the drift phase. The early
 // variant gains 8-10 % when a tile has several stale replicas (W >= 16 at p = 0.3) and costs 1-6 % when
 // it has about one or none, so both are built and the launch policy picks.
-template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED = false>
 __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPerSm)
     lossy_fused_tma_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
   constexpr int kConsumerWarps = CW;
@@ -194,11 +205,13 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   constexpr int kTile = TmaShape<CW>::kTile;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
-  // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) | stages
+  // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) |
+  //         stale masks per sub-packet of the PACKED build (kMaxStages x 64 B) | stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kTmaBarBytes - 4);
   StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + kTmaBarBytes);
-  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr);
+  PackedStale* pks = reinterpret_cast<PackedStale*>(smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr));
+  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale));
   const uint32_t S = G.stages;
   const uint32_t off_th = G.grad_slots * kTile * kGB;
   const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4, off_wire = off_v + kTile * 4;
@@ -230,56 +243,93 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     bool ok = true;
     const bool lh = G.hints & 1u;
     const uint64_t pol = policy_evict_first();
-    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
-      const uint32_t k = tile / G.tiles_per_packet;
-      const uint32_t c = tile - k * G.tiles_per_packet;
-      const uint32_t j = (P.k0 + k) / P.pps;
-      const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
-      const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
-      uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
-      packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale, gbad, pbad);
-      const uint32_t cnt = __popcll(recv);
-      if (c == 0 && lane == 0) {
-        if (P.count) P.count[k] = (uint8_t)cnt;
-        if (P.recv_bits) P.recv_bits[k] = recv;
-        if (P.stale_bits) P.stale_bits[k] = stale;
-        if (P.burst_out) {   // bursty loss: the packet's first tile stores its links' new states
-          P.burst_out[k] = gbad;
-          P.burst_out[(size_t)P.K + k] = pbad;
+    if constexpr (PACKED) {
+      // no masks here: every worker's piece of the tile is fetched, the compute warps decide what counts
+      for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+        const uint32_t kfirst = tile * G.packets_per_tile;
+        const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
+        const uint64_t e0 = (uint64_t)kfirst * P.P;
+        const uint32_t len = npk * P.P;
+        for (uint32_t g = 0; g < G.groups; ++g, ++it) {
+          const uint32_t s = it % S, par = (it / S) & 1u;
+          if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
+          const bool last = g + 1 == G.groups;
+          const uint32_t in_group = min((uint32_t)kGroup, W - g * kGroup);
+          unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+          if (lane == 0) {
+            StageHdr& h = hdrs[s];
+            h.recv = 0; h.stale = 0; h.e0 = e0; h.k = npk; h.len = len; h.cnt = 0; h.last = last ? 1u : 0u;
+            uint32_t bytes = in_group * len * kGB;
+            if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
+            mbar_arrive_expect_tx(full_bar(s), bytes);
+          }
+          __syncwarp();
+          if ((uint32_t)lane < in_group)
+            bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
+                     reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
+          if (last) {
+            if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
+            if constexpr (OPT == 1) {
+              if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s), lh, pol);
+              if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s), lh, pol);
+            }
+          }
+          armed_mask |= 1u << s;
+          armed_par = (armed_par & ~(1u << s)) | (par << s);
         }
       }
-      if constexpr (DRIFTK) {
-        for (uint32_t i = lane; i < W; i += 32)
-          if ((stale >> i) & 1ull)
-            bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
-      }
-      if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
-      for (uint32_t g = 0; g < G.groups; ++g, ++it) {
-        const uint32_t s = it % S, par = (it / S) & 1u;
-        if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
-        const bool last = g + 1 == G.groups;
-        const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
-        unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
-        if (lane == 0) {
-          StageHdr& h = hdrs[s];
-          h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
-          uint32_t bytes = __popc(bits) * len * kGB;
-          if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
-          mbar_arrive_expect_tx(full_bar(s), bytes);
-        }
-        __syncwarp();
-        if (lane < kGroup && ((bits >> lane) & 1u))
-          bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
-                   reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
-        if (last) {
-          if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
-          if constexpr (OPT == 1) {
-            if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s), lh, pol);
-            if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s), lh, pol);
+    } else {
+      for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+        const uint32_t k = tile / G.tiles_per_packet;
+        const uint32_t c = tile - k * G.tiles_per_packet;
+        const uint32_t j = (P.k0 + k) / P.pps;
+        const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
+        const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
+        uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
+        packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale, gbad, pbad);
+        const uint32_t cnt = __popcll(recv);
+        if (c == 0 && lane == 0) {
+          if (P.count) P.count[k] = (uint8_t)cnt;
+          if (P.recv_bits) P.recv_bits[k] = recv;
+          if (P.stale_bits) P.stale_bits[k] = stale;
+          if (P.burst_out) {   // bursty loss: the packet's first tile stores its links' new states
+            P.burst_out[k] = gbad;
+            P.burst_out[(size_t)P.K + k] = pbad;
           }
         }
-        armed_mask |= 1u << s;
-        armed_par = (armed_par & ~(1u << s)) | (par << s);
+        if constexpr (DRIFTK) {
+          for (uint32_t i = lane; i < W; i += 32)
+            if ((stale >> i) & 1ull)
+              bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
+        }
+        if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
+        for (uint32_t g = 0; g < G.groups; ++g, ++it) {
+          const uint32_t s = it % S, par = (it / S) & 1u;
+          if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
+          const bool last = g + 1 == G.groups;
+          const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
+          unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+          if (lane == 0) {
+            StageHdr& h = hdrs[s];
+            h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
+            uint32_t bytes = __popc(bits) * len * kGB;
+            if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
+            mbar_arrive_expect_tx(full_bar(s), bytes);
+          }
+          __syncwarp();
+          if (lane < kGroup && ((bits >> lane) & 1u))
+            bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
+                     reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
+          if (last) {
+            if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
+            if constexpr (OPT == 1) {
+              if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s), lh, pol);
+              if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s), lh, pol);
+            }
+          }
+          armed_mask |= 1u << s;
+          armed_par = (armed_par & ~(1u << s)) | (par << s);
+        }
       }
     }
     if (!ok || *abort_flag) {
@@ -309,9 +359,26 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u, sh_hint, pol);
             if (lane == 2) bulk_s2g(P.v + e0, smem_u32(st + off_v), len * 4u, sh_hint, pol);
           }
-          for (uint32_t i = lane; i < W; i += 32)
-            if (!((stale >> i) & 1ull))
-              bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB, sh_hint, pol);
+          if constexpr (PACKED) {
+            // replica i takes every run of consecutive sub-packets whose broadcast it received
+            const uint32_t npk = h.k;
+            for (uint32_t i = lane; i < W; i += 32) {
+              int run = -1;
+              for (uint32_t sp = 0; sp <= npk; ++sp) {
+                const bool fresh = sp < npk && !((pks[s].stale[sp < npk ? sp : 0] >> i) & 1ull);
+                if (fresh && run < 0) run = (int)sp;
+                if (!fresh && run >= 0) {
+                  bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0 + (uint64_t)run * P.P,
+                           smem_u32(st + off_wire + (size_t)run * P.P * kRB), (sp - (uint32_t)run) * P.P * kRB, sh_hint, pol);
+                  run = -1;
+                }
+              }
+            }
+          } else {
+            for (uint32_t i = lane; i < W; i += 32)
+              if (!((stale >> i) & 1ull))
+                bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB, sh_hint, pol);
+          }
           bulk_commit();
           bulk_wait_read0();          // shared memory of this stage may be overwritten after this
         }
@@ -327,11 +394,45 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     bool ok = true;
     float acc[kEpl];
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      // PACKED: this warp's 128 elements lie in one small packet; the warp evaluates that packet's masks
+      // itself, before it waits for the tile's data
+      uint64_t my_recv = 0, my_stale = 0;
+      uint32_t my_sp = 0;
+      bool my_first = false;
+      if constexpr (PACKED) {
+        const uint32_t kfirst = tile * G.packets_per_tile;
+        const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
+        const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;
+        if (widx < npk * P.P) {
+          my_sp = widx / P.P;
+          my_first = widx == my_sp * P.P;
+          const uint32_t k = kfirst + my_sp;
+          uint64_t gbad = 0, pbad = 0;
+          packet_masks<AGG | BCAST>(P, k, (P.k0 + k) / P.pps, lane, my_recv, my_stale, gbad, pbad);
+          if (my_first && lane == 0) {
+            if (P.count) P.count[k] = (uint8_t)__popcll(my_recv);
+            if (P.recv_bits) P.recv_bits[k] = my_recv;
+            if (P.stale_bits) P.stale_bits[k] = my_stale;
+            if (P.burst_out) {
+              P.burst_out[k] = gbad;
+              P.burst_out[(size_t)P.K + k] = pbad;
+            }
+          }
+          if constexpr (DRIFTK) {
+            uint64_t sm = my_stale;
+            while (sm) {
+              const int i = __ffsll((long long)sm) - 1;
+              sm &= sm - 1;
+              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + (uint64_t)kfirst * P.P + idx);
+            }
+          }
+        }
+      }
       for (uint32_t g = 0; g < G.groups; ++g, ++it) {
         const uint32_t s = it % S, par = (it / S) & 1u;
         if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
         const StageHdr& h = hdrs[s];
-        const uint64_t recv = h.recv;
+        const uint64_t recv = PACKED ? my_recv : h.recv;
         const uint32_t len = h.len;
         const bool active = idx < len;
         unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
@@ -356,8 +457,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           continue;
         }
         // ---- last group of the tile: estimate, update, wire value -----------------
-        const uint32_t cnt = h.cnt;
-        const uint64_t stale = h.stale, e0 = h.e0;
+        const uint32_t cnt = PACKED ? (uint32_t)__popcll(my_recv) : h.cnt;
+        const uint64_t stale = PACKED ? my_stale : h.stale, e0 = h.e0;
+        if constexpr (PACKED) {
+          if (my_first && lane == 0) pks[s].stale[my_sp] = my_stale;   // for the store warp, before this warp's arrive
+        }
         float wire[kEpl];
         // The first stale copies are requested now, so that their (L2) latency hides behind the arithmetic
         // below; they are used in the drift phase after this warp has handed the stage to the store warp.

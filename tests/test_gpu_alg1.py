@@ -22,6 +22,7 @@ CASES = [
     ("small_packets_register", 6, 256 * 90 + 24, 256, 0.3, 0.1, "adam", "bf16", "bf16", 0),
     ("zero_skip_on_drop", 4, 1024 * 33, 1024, 0.5, 0.2, "adam", "f32", "bf16", SKIP),
     ("tiny", 3, 45, 8, 0.5, 0.5, "sgd", "bf16", "bf16", 0),
+    ("packed_small_packets_low_loss", 8, 256 * 70 + 24, 256, 0.1, 0.1, "adam", "bf16", "bf16", 0),
 ]
 
 

@@ -20,6 +20,7 @@ CASES = [
     ("w40_self_lossless", 40, 1024 * 21, 1024, (0.3, 0.5), "sgd", "bf16", "f32", L.LOSSY_SELF_LOSSLESS, False),
     ("small_packets", 5, 256 * 77 + 8, 256, (0.1, 0.2), "adam", "bf16", "bf16", 0, False),
     ("always_leave", 4, 1024 * 12, 1024, (0.5, 1.0), "sgd", "f32", "bf16", 0, False),
+    ("packed_128", 6, 128 * 60, 128, (0.05, 0.5), "adam", "bf16", "bf16", 0, False),
     ("alg1_one_chain_per_packet", 8, 2048 * 33, 2048, (0.1, 0.3), "adam", "bf16", "bf16", 0, True),
 ]
 

@@ -92,6 +92,11 @@ EDGE = [
     ("bulk_packed_512_w3_f32", 3, 512 * 21, 512, 0.4, "adam", "f32", "f32", SKIP),
     ("bulk_packed_1024_w16", 16, 1024 * 9 + 512, 1024, 0.1, "adam", "bf16", "bf16", LOSSLESS),
     ("bulk_packed_256_heavy_loss", 8, 256 * 64, 256, 0.6, "adam", "bf16", "bf16", 0),
+    ("packed_wide_8_per_tile_low_loss", 16, 256 * 61 + 40, 256, 0.1, "adam", "bf16", "bf16", 0),
+    ("packed_wide_4_per_tile_f32", 5, 512 * 27, 512, 0.15, "adam", "f32", "f32", SKIP),
+    ("packed_twin_w24_two_per_tile", 24, 512 * 45 + 8, 512, 0.05, "sgd", "bf16", "bf16", 0),
+    ("packed_128_elements_any_loss", 40, 128 * 90, 128, 0.4, "adam", "bf16", "f32", LOSSLESS),
+    ("packed_128_w4", 4, 128 * 33 + 16, 128, 0.1, "sgd", "f32", "bf16", 0),
 ]
 
 
