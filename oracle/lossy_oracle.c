@@ -383,3 +383,28 @@ int NAME(packet_sqnorms)(const oracle_config* c, uint64_t n_slab, const void* co
     }
   return 0;
 }
+
+/*
+ * Delivery indicators alone (Section 3's s and r for independent loss), for `packets` packets starting at
+ * bucket packet k0: recv bit i = worker i's piece reached the owner, stale bit i = replica i missed the
+ * broadcast, count = received pieces. Lets a test compare EVERY packet of a full-size bucket.
+ */
+int NAME(masks)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t packets, uint64_t* recv_bits,
+                uint64_t* stale_bits, uint8_t* count) {
+  if (!c || !recv_bits || !stale_bits || !count) return 1;
+  const uint32_t Tg = NAME(threshold)(c->p_grad), Tp = NAME(threshold)(c->p_param);
+  for (uint64_t kl = 0; kl < packets; ++kl) {
+    const uint64_t k = k0 + kl, kg = c->packet_base + k;
+    const uint32_t j = NAME(owner)(c, k);
+    uint64_t recv = 0, stale = 0;
+    uint32_t cnt = 0;
+    for (uint32_t i = 0; i < c->W; ++i) {
+      int s = NAME(hash_u32)(c->seed, step, i, j, kg) >= Tg;
+      if ((c->flags & FLAG_SELF_LOSSLESS) && i == j) s = 1;
+      if (s) { recv |= 1ULL << i; ++cnt; }
+      if (i != j && NAME(hash_u32)(c->seed, step, j, i, kg) < Tp) stale |= 1ULL << i;
+    }
+    recv_bits[kl] = recv; stale_bits[kl] = stale; count[kl] = (uint8_t)cnt;
+  }
+  return 0;
+}

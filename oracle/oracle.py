@@ -82,6 +82,9 @@ def _lib(f64: bool):
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
         ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
+        mk = getattr(lib, pre + "masks")
+        mk.restype = C.c_int
+        mk.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
         sq = getattr(lib, pre + "packet_sqnorms")
         sq.restype = C.c_int
         sq.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p]
@@ -169,6 +172,19 @@ class Oracle:
 
     def set_lr(self, lr: float) -> None:
         self.cfg.lr = lr
+
+    def masks(self, t, k0=0, packets=None):
+        """(recv_bits, stale_bits, count) of `packets` packets from bucket packet k0 at step t (independent loss)."""
+        K = (self.n + self.P - 1) // self.P
+        packets = K - k0 if packets is None else packets
+        recv = np.zeros(packets, np.uint64)
+        stale = np.zeros(packets, np.uint64)
+        count = np.zeros(packets, np.uint8)
+        rc = getattr(self.lib, self.pre + "masks")(C.byref(self.cfg), t, k0, packets, _ptr(recv), _ptr(stale),
+                                                   _ptr(count))
+        if rc != 0:
+            raise ValueError("oracle_masks rejected its arguments")
+        return recv, stale, count
 
     def packet_sqnorms(self, grads):
         """[W][packets] squared norms of the gradient pieces, in double."""

@@ -39,6 +39,11 @@ def _run_full(w, steps, slab_packets, n_random, full_drift):
         gd = [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)]
         gpu.step_fused(t, gd)                       # the call bench.py times (with every optional output)
         out = gpu.outputs()
+        # masks, received counts and stale sets of EVERY packet of the bucket, bit for bit
+        recv_all, stale_all, count_all = oracles[0][3].masks(t, 0, w.K)
+        assert_same(out["recv_bits"], recv_all, f"{w.name} step {t} recv_bits of all {w.K} packets")
+        assert_same(out["stale_bits"], stale_all, f"{w.name} step {t} stale_bits of all {w.K} packets")
+        assert_same(out["count"], count_all, f"{w.name} step {t} counts of all {w.K} packets")
         for k0, e0, e1, orc in oracles:
             ref = orc.step(t, [to_np(g[e0:e1]) for g in gd])
             k1 = k0 + orc.packets

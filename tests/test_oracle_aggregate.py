@@ -215,3 +215,17 @@ def test_slab_by_slab_equals_whole_bucket():
                 assert np.array_equal(o.replicas[i], whole.replicas[i][e0:e1])
             tot += r["sumsq"]
         assert np.allclose(tot, rw["sumsq"], rtol=1e-12)
+
+
+def test_mask_only_routine_agrees_with_the_step():
+    W, P, K = 7, 8, 500
+    n = P * K - 3
+    o = _mk(W, n, P, 0.3, seed=21, flags=oracle.SELF_LOSSLESS, packet_base=77)
+    g = _rand_grads(np.random.default_rng(0), W, n)
+    for t in (1, 2, 9):
+        r = o.step(t, g)
+        recv, stale, count = o.masks(t)
+        assert np.array_equal(recv, r["recv_bits"]) and np.array_equal(stale, r["stale_bits"])
+        assert np.array_equal(count, r["count"])
+        recv2, stale2, count2 = o.masks(t, k0=100, packets=50)
+        assert np.array_equal(recv2, recv[100:150]) and np.array_equal(stale2, stale[100:150])
