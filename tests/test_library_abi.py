@@ -60,3 +60,29 @@ def test_product_path_never_touches_the_oracle():
     for f in ("lossy_oracle.c", "oracle.py"):
         src = open(os.path.join(ROOT, "oracle", f)).read()
         assert "paper_2507_07114_b200" not in src and "lossy.h" not in src
+
+
+def test_configuration_is_validated_on_the_host_before_any_cuda_call():
+    """Bad configurations are rejected with LOSSY_EINVAL by plain host code, so this runs without a GPU."""
+    lib = L.load_library()
+    good = dict(W=8, packet_elems=2048, n=2048 * 10, packet_base=0, p_grad=0.1, p_param=0.1, seed=0,
+                grad_dtype=L.LOSSY_BF16, replica_dtype=L.LOSSY_BF16, optimizer=L.LOSSY_ADAM, flags=0,
+                lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, shard_packet0=0, bucket_packets=0)
+    bad = [dict(W=0), dict(W=65), dict(packet_elems=0), dict(packet_elems=100), dict(p_grad=1.0),
+           dict(p_param=-1e-9), dict(p_grad=float("nan")), dict(grad_dtype=2), dict(replica_dtype=7),
+           dict(optimizer=2), dict(flags=64), dict(n=2 ** 40, packet_elems=8),          # more than 2^31 chunks
+           dict(shard_packet0=1), dict(shard_packet0=8, bucket_packets=12),             # range leaves the bucket
+           dict(n=2048 * 10 - 8, bucket_packets=20)]                                    # ragged range inside a bucket
+    for change in bad:
+        kw = dict(good)
+        kw.update(change)
+        cfg = L.lossy_config(**kw)
+        ctx = ctypes.c_void_p()
+        assert lib.lossy_init(ctypes.byref(cfg), ctypes.byref(ctx)) == L.LOSSY_EINVAL, change
+        assert not ctx.value
+    assert lib.lossy_init(None, None) == L.LOSSY_EINVAL
+    # entry points refuse a NULL context instead of dereferencing it
+    assert lib.lossy_set_lr(None, 0.1) == L.LOSSY_EINVAL
+    assert lib.lossy_device_status(None, None) == L.LOSSY_EINVAL
+    assert lib.lossy_last_error(None) == b"NULL context"
+    lib.lossy_destroy(None)
