@@ -201,6 +201,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--configs", default="1,2,3,5")
     ap.add_argument("--steps", type=int, default=0, help="0 = each configuration's own step count")
+    ap.add_argument("--elements", type=int, default=0, help="unfused: bucket size override (small case for profiling)")
     args = ap.parse_args()
     cfg = workload.baseline_workloads()
     want = set(args.configs.split(","))
@@ -223,7 +224,10 @@ def main():
         # the full model (32 layers) needs 189 GB resident and does not fit one GPU: 24 layers + embedding + head
         print(json.dumps(run_model_streamed(cfg["cfg4_w8_full_model"], 24, args.steps or 20)), flush=True)
     if "unfused" in want:
-        for r in run_unfused(cfg["cfg2_w8_layer_adam"]):
+        base2 = cfg["cfg2_w8_layer_adam"]
+        if args.elements:
+            base2 = workload.scaled(base2, args.elements)
+        for r in run_unfused(base2, steps=args.steps or 20):
             print(json.dumps(r), flush=True)
     if "alg1" in want:
         # Algorithm 1 mode on the config-2 bucket: packet-granular and shard-granular (P = n / W) drops
