@@ -12,6 +12,12 @@
 // the broadcast are not written; their old packet is read (L2-prefetched by the producer) only to
 // accumulate the drift term. No cluster launch and no multicast: the path has no cross-CTA reuse.
 //
+// Template variants, picked per context by the host's launch policy: CW (compute warps: 16 = one CTA per
+// SM with 2048-element tiles, 8 = two CTAs per SM with 1024-element tiles), GS (workers per pipeline stage, 4
+// or 8), PRE (registers per lane for stale replica data requested before the tile's arithmetic, 0 or 16) and
+// PACKED (packets shorter than a tile: several whole packets per tile, masks evaluated by the compute warps).
+// Drift norms are finalised by the last CTA to finish (fence + ticket counter; nothing waits on another CTA).
+//
 // Every wait on an mbarrier is bounded: after kMaxPolls unsuccessful polls the CTA raises a
 // shared abort flag, records a code in the context's device status word and every role leaves
 // its loop; the producer then gives its own copies in flight a bounded time to land.
