@@ -8,7 +8,7 @@
 
 #include <new>
 
-#include "lossy_tma.cuh"
+#include "lossy_phase_tma.cuh"
 
 using namespace lossy;
 
@@ -204,7 +204,7 @@ int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t
 
 template <int CW, int GS, int PRE = 0, bool PACKED = false>
 int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
-  TmaGeom G;
+  TmaGeom G = {};
   if (!tma_geometry<CW, GS, PACKED>(ctx, G)) return LOSSY_OK;
   *used = true;
   // without drift norms nothing reads the stale copies: the plain build serves
@@ -290,6 +290,123 @@ int dispatch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks) 
     if (!gb && rb) return adam ? launch<PH, F32, BF16, 1>(ctx, P, s, blocks) : launch<PH, F32, BF16, 0>(ctx, P, s, blocks);
     return adam ? launch<PH, F32, F32, 1>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
   }
+}
+
+
+// ---- the single-phase calls through the bulk-copy pipeline ---------------------------------
+constexpr uint32_t kPhaseSmemFixed = kTmaBarBytes + kPhaseMaxStages * sizeof(StageHdr);
+
+template <int PH, int CW, int GS>
+bool phase_geometry(const lossy_ctx* ctx, TmaGeom& G) {
+  constexpr uint32_t kTile = TmaShape<CW>::kTile;
+  constexpr bool kGrouped = PH == AGG || PH == DRIFT;
+  const lossy_config& c = ctx->cfg;
+  const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
+  if (kfull == 0 || kfull >= (1ull << 31) || c.packet_elems < kTile) return false;
+  memset(&G, 0, sizeof G);
+  G.packets_per_tile = 1;
+  G.full_packets = (uint32_t)kfull;
+  const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
+  const uint32_t eb = PH == AGG ? gb : PH == STEP ? 4u : rb;
+  G.grad_slots = kGrouped ? (c.W < (uint32_t)GS ? c.W : (uint32_t)GS) : 0u;
+  G.groups = kGrouped ? (c.W + GS - 1) / GS : 1u;
+  G.stage_bytes = (phase_stage_bytes<PH>(kTile, G.grad_slots, eb, c.optimizer == LOSSY_ADAM) + 127u) & ~127u;
+  const uint32_t budget = tma_smem_budget<CW>(ctx);
+  if (budget < kPhaseSmemFixed + 2 * G.stage_bytes) return false;
+  G.stages = (budget - kPhaseSmemFixed) / G.stage_bytes;
+  if (G.stages > (uint32_t)kPhaseMaxStages) G.stages = kPhaseMaxStages;
+  // the optimizer step reads and writes equal amounts: deeper than three stages its loads run too far ahead
+  // of its stores (measured 1.01 of the copy rate with three stages, 0.90 with seven)
+  if (PH == STEP && G.stages > 3u) G.stages = 3u;
+  G.tiles_per_packet = (c.packet_elems + kTile - 1) / kTile;
+  const uint64_t tiles = kfull * G.tiles_per_packet;
+  if (tiles >= (1ull << 31)) return false;
+  G.num_tiles = (uint32_t)tiles;
+  G.status = ctx->status;
+  G.hints = 0;
+  return true;
+}
+
+template <int PH, class T, int OPT, int CW, int GS>
+int launch_phase_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
+  auto kern = lossy_phase_tma_kernel<PH, T, OPT, CW, GS>;
+  const uint32_t smem = kPhaseSmemFixed + G.stages * G.stage_bytes;
+  uint32_t blocks = (uint32_t)(ctx->num_sms * TmaShape<CW>::kCtasPerSm);
+  if (blocks > G.num_tiles) blocks = G.num_tiles;
+  *blocks_out = blocks;
+  if (ctx->plan_only) return LOSSY_OK;
+  static bool opted_in[kMaxDevices];   // per kernel instantiation and device: raise the dynamic shared memory limit once
+  cudaError_t e;
+  if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
+    if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
+    if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+  }
+  kern<<<blocks, TmaShape<CW>::kThreads, smem, s>>>(P, G);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "bulk-copy kernel launch", e);
+  ctx->launches++;
+  return LOSSY_OK;
+}
+
+template <int PH, int CW, int GS>
+int try_phase_tma(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks, bool* used) {
+  TmaGeom G;
+  if (!phase_geometry<PH, CW, GS>(ctx, G)) return LOSSY_OK;
+  *used = true;
+  const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
+  if constexpr (PH == AGG) {
+    return ctx->cfg.grad_dtype == LOSSY_BF16 ? launch_phase_tma<PH, BF16, 0, CW, GS>(ctx, P, G, s, blocks)
+                                             : launch_phase_tma<PH, F32, 0, CW, GS>(ctx, P, G, s, blocks);
+  } else if constexpr (PH == STEP) {
+    return adam ? launch_phase_tma<PH, F32, 1, CW, GS>(ctx, P, G, s, blocks)
+                : launch_phase_tma<PH, F32, 0, CW, GS>(ctx, P, G, s, blocks);
+  } else {
+    return ctx->cfg.replica_dtype == LOSSY_BF16 ? launch_phase_tma<PH, BF16, 0, CW, GS>(ctx, P, G, s, blocks)
+                                                : launch_phase_tma<PH, F32, 0, CW, GS>(ctx, P, G, s, blocks);
+  }
+}
+
+// One single-phase call: complete packets through the bulk-copy pipeline where a build fits (packets of at
+// least one tile, not Algorithm 1's aggregate), a ragged last packet or everything else through the register
+// kernel. With drift norms, pass 0 only sizes the grids: the blocks of both launches draw tickets from one
+// counter and the last of them finalises the norms.
+template <int PH>
+int run_phase(lossy_ctx* ctx, const Params& P, float* norms, double* sumsq, cudaStream_t s) {
+  const lossy_config& c = ctx->cfg;
+  const bool bulk = !(c.flags & LOSSY_REGISTER_PATH) && !P.ghat_prev;
+  // wide tiles (one CTA per SM) when they divide the packet and the streamed arrays fit two groups
+  const bool wide = c.packet_elems % TmaShape<16>::kTile == 0 && c.W <= 16;
+  uint32_t tma_blocks = 0, tail_blocks = 0;
+  for (int pass = PH == DRIFT ? 0 : 1; pass < 2; ++pass) {
+    ctx->plan_only = pass == 0;
+    Params Q = P;
+    if (PH == DRIFT && pass == 1) {
+      Q.ticket = ctx->ticket;
+      Q.total_rows = tma_blocks + tail_blocks;
+      Q.norms = norms;
+      Q.sumsq = sumsq;
+    }
+    bool used = false;
+    int rc = LOSSY_OK;
+    if (bulk) {
+      if (wide) rc = try_phase_tma<PH, 16, 8>(ctx, Q, s, &tma_blocks, &used);
+      if (!rc && !used) rc = try_phase_tma<PH, 8, 8>(ctx, Q, s, &tma_blocks, &used);
+    }
+    if (!rc) {
+      if (used) {
+        Q.chunk_begin = (uint32_t)((c.n / c.packet_elems) * ctx->chunks_per_packet);
+        Q.partials_row0 = tma_blocks;
+      } else {
+        tma_blocks = 0;
+      }
+      if (Q.chunk_begin < Q.num_chunks) rc = dispatch<PH>(ctx, Q, s, &tail_blocks);
+      else tail_blocks = 0;
+    }
+    ctx->plan_only = false;
+    if (rc) return rc;
+  }
+  return LOSSY_OK;
 }
 
 }  // namespace
@@ -418,7 +535,7 @@ static int aggregate_impl(lossy_ctx* ctx, uint64_t step, const void* const* grad
   P.ghat_prev = ghat_prev;
   P.count = count;
   P.recv_bits = recv_bits;
-  return dispatch<AGG>(ctx, P, (cudaStream_t)stream, nullptr);
+  return run_phase<AGG>(ctx, P, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat, uint8_t* count,
@@ -457,7 +574,7 @@ int lossy_step(lossy_ctx* ctx, uint64_t step, const float* ghat, const uint8_t* 
   P.master = master;
   P.m = m;
   P.v = v;
-  return dispatch<STEP>(ctx, P, (cudaStream_t)stream, nullptr);
+  return run_phase<STEP>(ctx, P, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master, void* const* replicas, uint64_t* stale_bits,
@@ -471,7 +588,7 @@ int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master, void* co
   for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.replicas[i] = replicas[i];
   P.master = const_cast<float*>(master);
   P.stale_bits = stale_bits;
-  return dispatch<BCAST>(ctx, P, (cudaStream_t)stream, nullptr);
+  return run_phase<BCAST>(ctx, P, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas, float* norms, double* sumsq,
@@ -490,17 +607,7 @@ int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas
   fill_common(ctx, 1, P);
   for (uint32_t i = 0; i < ctx->cfg.W; ++i) P.replicas[i] = const_cast<void*>(replicas[i]);
   P.master = const_cast<float*>(master);
-  // grid size first, so that the kernel knows how many blocks will draw a ticket; the last one finalises
-  uint32_t blocks = 0;
-  ctx->plan_only = true;
-  int rc = dispatch<DRIFT>(ctx, P, (cudaStream_t)stream, &blocks);
-  ctx->plan_only = false;
-  if (rc) return rc;
-  P.ticket = ctx->ticket;
-  P.total_rows = blocks;
-  P.norms = norms;
-  P.sumsq = sumsq;
-  return dispatch<DRIFT>(ctx, P, (cudaStream_t)stream, &blocks);
+  return run_phase<DRIFT>(ctx, P, norms, sumsq, (cudaStream_t)stream);
 }
 
 static int fused_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* master,

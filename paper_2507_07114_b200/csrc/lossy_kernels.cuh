@@ -22,13 +22,13 @@ __device__ __forceinline__ void divide_by_count(float (&a)[N], uint32_t cnt) {
   }
 }
 
-// One optimizer update of 8 elements, every operation rounded on its own
+// One optimizer update of N elements, every operation rounded on its own
 // (Section 3 step (3); Adam as bias-corrected Kingma-Ba with host-side corrections).
-template <int OPT>
-__device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8], float (&th)[8], float (&m)[8],
-                                           float (&v)[8]) {
+template <int OPT, int N>
+__device__ __forceinline__ void optimizer_n(const Params& P, const float (&g)[N], float (&th)[N], float (&m)[N],
+                                            float (&v)[N]) {
 #pragma unroll
-  for (int x = 0; x < 8; ++x) {
+  for (int x = 0; x < N; ++x) {
     if constexpr (OPT == 0) {
       th[x] = __fsub_rn(th[x], __fmul_rn(P.lr, g[x]));
     } else {
@@ -42,6 +42,11 @@ __device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8],
       v[x] = vn;
     }
   }
+}
+template <int OPT>
+__device__ __forceinline__ void optimizer8(const Params& P, const float (&g)[8], float (&th)[8], float (&m)[8],
+                                           float (&v)[8]) {
+  optimizer_n<OPT, 8>(P, g, th, m, v);
 }
 
 // Last-block drift finalisation. Every block has stored its row of `partials`; the block that draws the
