@@ -144,6 +144,53 @@ __device__ __forceinline__ void packet_masks(const Params& P, uint32_t k, uint32
   packet_masks<PH>(P, k, j, lane, recv, stale, gbad, pbad);
 }
 
+// The same draws for several packets per ballot (W <= 32, not Algorithm 1's aggregate): the warp's lanes
+// are split into 32 / Wp segments of Wp lanes (Wp = W rounded up to a power of two); a lane evaluates
+// link `i` of the packet `k` (owner `j`) of its segment. One warp evaluating one packet at a time is a
+// chain of dependent instructions (the hash) that bounds a producer warp when tiles carry few bytes.
+struct BatchDraws {
+  uint32_t recv_ok;     // bit = gradient piece delivered
+  uint32_t grad_lost;   // bit = gradient link in its lossy state (before the reliable channel)
+  uint32_t bcast_lost;  // bit = replica missed the broadcast (before the reliable channel)
+};
+template <int PH>
+__device__ __forceinline__ BatchDraws batch_draws(const Params& P, uint32_t k, uint32_t j, uint32_t i, bool valid) {
+  const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k);
+  const bool bursty = P.burst_in != nullptr;
+  BatchDraws d = {0u, 0u, 0u};
+  if constexpr (PH & AGG) {
+    const bool was = bursty && ((P.burst_in[k] >> i) & 1ull);
+    const uint32_t u = pair_hash(pkey, i, j);
+    bool lost = bursty ? (was ? u < P.Tstay : u < P.Tenter) : u < P.Tg;
+    if ((P.flags & 1u) && i == j) lost = false;
+    d.recv_ok = __ballot_sync(0xFFFFFFFFu, valid && !lost);
+    d.grad_lost = __ballot_sync(0xFFFFFFFFu, valid && lost);
+  }
+  if constexpr (PH & BCAST) {
+    const bool was = bursty && ((P.burst_in[(size_t)P.K + k] >> i) & 1ull);
+    const uint32_t u = pair_hash(pkey, j, i);
+    const bool lost = i != j && (bursty ? (was ? u < P.Tstay : u < P.Tenter) : u < P.Tp);
+    d.bcast_lost = __ballot_sync(0xFFFFFFFFu, valid && lost);
+  }
+  return d;
+}
+// masks of the packet `k` whose segment starts at lane `src` (segment mask `wmask`), as packet_masks returns them
+template <int PH>
+__device__ __forceinline__ void batch_masks(const Params& P, const BatchDraws& d, uint32_t k, int src, uint32_t wmask,
+                                            uint64_t& recv, uint64_t& stale, uint64_t& gbad, uint64_t& pbad) {
+  recv = stale = gbad = pbad = 0;
+  if constexpr (PH & AGG) {
+    recv = (d.recv_ok >> src) & wmask;
+    gbad = (d.grad_lost >> src) & wmask;
+    if (P.reliable) recv |= P.reliable[k] & ((1ull << P.W) - 1ull);   // W <= 32 here
+  }
+  if constexpr (PH & BCAST) {
+    stale = (d.bcast_lost >> src) & wmask;
+    pbad = stale;
+    if (P.reliable) stale &= ~P.reliable[(size_t)P.K + k];
+  }
+}
+
 template <int PH, class GT, class RT, int OPT>
 __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const __grid_constant__ Params P) {
   const int lane = threadIdx.x & 31;

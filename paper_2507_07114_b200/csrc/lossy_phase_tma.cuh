@@ -114,7 +114,6 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     const uint32_t B = 32u >> lgWp;                                // tiles per batch
     const uint32_t wmask = Wp == 32 ? 0xFFFFFFFFu : ((1u << Wp) - 1u);
     const uint64_t all = W == 64 ? ~0ull : ((1ull << W) - 1ull);
-    const bool bursty = P.burst_in != nullptr;
     for (uint32_t tile0 = blockIdx.x; ok && tile0 < G.num_tiles; tile0 += B * gridDim.x) {
       // this lane's tile of the batch and its worker there
       const uint32_t b_l = (uint32_t)lane >> lgWp, i_l = (uint32_t)lane & (Wp - 1u);
@@ -123,20 +122,9 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       const uint32_t k_l = tv ? tile_l / G.tiles_per_packet : 0u;
       const uint32_t c_l = tv ? tile_l - k_l * G.tiles_per_packet : 0u;
       const uint32_t j_l = (P.k0 + k_l) / P.pps;
-      uint32_t ok_all = 0, lost_all = 0;     // W <= 32: one bit per (tile of the batch, worker)
+      BatchDraws draws = {0u, 0u, 0u};         // W <= 32: one bit per (tile of the batch, worker)
       if constexpr (kMasked) {
-        if (W <= 32) {
-          const uint64_t pkey = packet_key_of(P.step_key, P.packet_base + k_l);
-          const uint64_t was_bits = bursty ? P.burst_in[(PH == BCAST ? (size_t)P.K : 0) + k_l] : 0ull;
-          const bool was = (was_bits >> i_l) & 1ull;
-          const uint32_t u = PH == AGG ? pair_hash(pkey, i_l, j_l) : pair_hash(pkey, j_l, i_l);
-          bool lost = bursty ? (was ? u < P.Tstay : u < P.Tenter) : u < (PH == AGG ? P.Tg : P.Tp);
-          if (PH == AGG && (P.flags & 1u) && i_l == j_l) lost = false;   // the owner's own piece stays on the node
-          if (PH == BCAST && i_l == j_l) lost = false;                    // the owner holds the new value
-          const bool valid = tv && i_l < W;
-          ok_all = __ballot_sync(0xFFFFFFFFu, valid && !lost);
-          lost_all = __ballot_sync(0xFFFFFFFFu, valid && lost);
-        }
+        if (W <= 32) draws = batch_draws<PH>(P, k_l, j_l, i_l, tv && i_l < W);
       }
       for (uint32_t b = 0; ok && b < B; ++b) {
         const uint32_t tile = tile0 + b * gridDim.x;
@@ -151,16 +139,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         uint32_t cnt = 1;
         if constexpr (kMasked) {
           if (W <= 32) {
-            const uint64_t okb = (ok_all >> src) & wmask, lostb = (lost_all >> src) & wmask;
-            if constexpr (PH == AGG) {
-              recv = okb;
-              gbad = lostb;
-              if (P.reliable) recv |= P.reliable[k] & all;          // the reliable channel always delivers
-            } else {
-              stale = lostb;
-              pbad = lostb;
-              if (P.reliable) stale &= ~P.reliable[(size_t)P.K + k];
-            }
+            batch_masks<PH>(P, draws, k, src, wmask, recv, stale, gbad, pbad);
           } else {
             packet_masks<PH>(P, k, j, lane, recv, stale, gbad, pbad);
           }
@@ -224,10 +203,10 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     }
     if (!ok || *abort_flag) {
       // give this CTA's copies in flight a bounded time to land before the CTA exits
-      for (uint32_t s = 0; s < S; ++s)
-        if ((armed_mask >> s) & 1u)
+      for (uint32_t q = 0; q < S; ++q)
+        if ((armed_mask >> q) & 1u)
           for (uint32_t i = 0; i < (1u << 16); ++i)
-            if (mbar_try_wait(full_bar(s), (armed_par >> s) & 1u)) break;
+            if (mbar_try_wait(full_bar(q), (armed_par >> q) & 1u)) break;
     }
   } else if (warp == kConsumerWarps + 1) {
     // ================================ store warp =================================

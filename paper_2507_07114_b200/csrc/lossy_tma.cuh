@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
 
   if (warp == kConsumerWarps) {
     // =============================== producer warp ===============================
-    uint32_t it = 0, armed_mask = 0, armed_par = 0;
+    uint32_t s = 0, par = 0, armed_mask = 0, armed_par = 0;
     bool ok = true;
     const bool lh = G.hints & 1u;
     const uint64_t pol = policy_evict_first();
@@ -257,8 +257,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
         const uint64_t e0 = (uint64_t)kfirst * P.P;
         const uint32_t len = npk * P.P;
-        for (uint32_t g = 0; g < G.groups; ++g, ++it) {
-          const uint32_t s = it % S, par = (it / S) & 1u;
+        for (uint32_t g = 0; g < G.groups; ++g) {
           if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
           const bool last = g + 1 == G.groups;
           const uint32_t in_group = min((uint32_t)kGroup, W - g * kGroup);
@@ -283,78 +282,101 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           }
           armed_mask |= 1u << s;
           armed_par = (armed_par & ~(1u << s)) | (par << s);
+          if (++s == S) { s = 0; par ^= 1u; }
         }
       }
     } else {
-      for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
-        const uint32_t k = tile / G.tiles_per_packet;
-        const uint32_t c = tile - k * G.tiles_per_packet;
-        const uint32_t j = (P.k0 + k) / P.pps;
-        const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
-        const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
-        uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
-        packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale, gbad, pbad);
-        const uint32_t cnt = __popcll(recv);
-        if (c == 0 && lane == 0) {
-          if (P.count) P.count[k] = (uint8_t)cnt;
-          if (P.recv_bits) P.recv_bits[k] = recv;
-          if (P.stale_bits) P.stale_bits[k] = stale;
-          if (P.burst_out) {   // bursty loss: the packet's first tile stores its links' new states
-            P.burst_out[k] = gbad;
-            P.burst_out[(size_t)P.K + k] = pbad;
-          }
-        }
-        if constexpr (DRIFTK) {
-          for (uint32_t i = lane; i < W; i += 32)
-            if ((stale >> i) & 1ull)
-              bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
-        }
-        if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
-        for (uint32_t g = 0; g < G.groups; ++g, ++it) {
-          const uint32_t s = it % S, par = (it / S) & 1u;
-          if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
-          const bool last = g + 1 == G.groups;
-          const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
-          unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
-          if (lane == 0) {
-            StageHdr& h = hdrs[s];
-            h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
-            uint32_t bytes = __popc(bits) * len * kGB;
-            if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
-            mbar_arrive_expect_tx(full_bar(s), bytes);
-          }
-          __syncwarp();
-          if (lane < kGroup && ((bits >> lane) & 1u))
-            bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
-                     reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
-          if (last) {
-            if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
-            if constexpr (OPT == 1) {
-              if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s), lh, pol);
-              if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s), lh, pol);
+      // The delivery draws are taken for a batch of tiles per ballot where the lanes allow it (W <= 16, not
+      // Algorithm 1): one warp hashing one packet at a time is a chain of dependent instructions that would
+      // bound the CTA when a tile carries few bytes.
+      uint32_t Wp = 32;
+      if (W <= 16 && !P.ghat_prev) { Wp = 1; while (Wp < W) Wp <<= 1; }
+      const uint32_t lgWp = 31u - (uint32_t)__clz((int)Wp);
+      const uint32_t B = 32u >> lgWp;                                // tiles per batch
+      const uint32_t wmask = Wp == 32 ? 0xFFFFFFFFu : ((1u << Wp) - 1u);
+      for (uint32_t tile0 = blockIdx.x; ok && tile0 < G.num_tiles; tile0 += B * gridDim.x) {
+        const uint32_t b_l = (uint32_t)lane >> lgWp, i_l = (uint32_t)lane & (Wp - 1u);
+        const uint32_t tile_l = tile0 + b_l * gridDim.x;
+        const bool tv = tile_l < G.num_tiles;
+        const uint32_t k_l = tv ? tile_l / G.tiles_per_packet : 0u;
+        const uint32_t c_l = tv ? tile_l - k_l * G.tiles_per_packet : 0u;
+        const uint32_t j_l = (P.k0 + k_l) / P.pps;
+        BatchDraws draws = {0u, 0u, 0u};
+        if (B > 1) draws = batch_draws<AGG | BCAST>(P, k_l, j_l, i_l, tv && i_l < W);
+        for (uint32_t b = 0; ok && b < B; ++b) {
+          const uint32_t tile = tile0 + b * gridDim.x;
+          if (tile >= G.num_tiles) break;
+          const int src = (int)(b * Wp);
+          const uint32_t k = __shfl_sync(0xFFFFFFFFu, k_l, src);
+          const uint32_t c = __shfl_sync(0xFFFFFFFFu, c_l, src);
+          const uint32_t j = __shfl_sync(0xFFFFFFFFu, j_l, src);
+          const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
+          const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
+          uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
+          if (B > 1) batch_masks<AGG | BCAST>(P, draws, k, src, wmask, recv, stale, gbad, pbad);
+          else packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale, gbad, pbad);
+          const uint32_t cnt = __popcll(recv);
+          if (c == 0 && lane == 0) {
+            if (P.count) P.count[k] = (uint8_t)cnt;
+            if (P.recv_bits) P.recv_bits[k] = recv;
+            if (P.stale_bits) P.stale_bits[k] = stale;
+            if (P.burst_out) {   // bursty loss: the packet's first tile stores its links' new states
+              P.burst_out[k] = gbad;
+              P.burst_out[(size_t)P.K + k] = pbad;
             }
           }
-          armed_mask |= 1u << s;
-          armed_par = (armed_par & ~(1u << s)) | (par << s);
+          if constexpr (DRIFTK) {
+            for (uint32_t i = lane; i < W; i += 32)
+              if ((stale >> i) & 1ull)
+                bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
+          }
+          if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
+          for (uint32_t g = 0; g < G.groups; ++g) {
+            if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
+            const bool last = g + 1 == G.groups;
+            const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
+            unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+            if (lane == 0) {
+              StageHdr& h = hdrs[s];
+              h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
+              uint32_t bytes = __popc(bits) * len * kGB;
+              if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
+              mbar_arrive_expect_tx(full_bar(s), bytes);
+            }
+            __syncwarp();
+            if (lane < kGroup && ((bits >> lane) & 1u))
+              bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
+                       reinterpret_cast<const typename GT::raw*>(P.grads[g * kGroup + lane]) + e0, len * kGB, full_bar(s), lh, pol);
+            if (last) {
+              if (lane == 8) bulk_g2s(smem_u32(st + off_th), P.master + e0, len * 4u, full_bar(s), lh, pol);
+              if constexpr (OPT == 1) {
+                if (lane == 9) bulk_g2s(smem_u32(st + off_m), P.m + e0, len * 4u, full_bar(s), lh, pol);
+                if (lane == 10) bulk_g2s(smem_u32(st + off_v), P.v + e0, len * 4u, full_bar(s), lh, pol);
+              }
+            }
+            armed_mask |= 1u << s;
+            armed_par = (armed_par & ~(1u << s)) | (par << s);
+            if (++s == S) { s = 0; par ^= 1u; }
+          }
         }
       }
     }
     if (!ok || *abort_flag) {
       // give this CTA's copies in flight a bounded time to land before the CTA exits
-      for (uint32_t s = 0; s < S; ++s)
-        if ((armed_mask >> s) & 1u)
+      for (uint32_t q = 0; q < S; ++q)
+        if ((armed_mask >> q) & 1u)
           for (uint32_t i = 0; i < (1u << 16); ++i)
-            if (mbar_try_wait(full_bar(s), (armed_par >> s) & 1u)) break;
+            if (mbar_try_wait(full_bar(q), (armed_par >> q) & 1u)) break;
     }
   } else if (warp == kConsumerWarps + 1) {
     // ================================ store warp =================================
-    uint32_t it = 0;
+    uint32_t s = 0, par = 0;
     bool ok = true;
     const bool sh_hint = G.hints & 2u;
     const uint64_t pol = policy_evict_first();
+    auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
-      for (uint32_t g = 0; g < G.groups; ++g, ++it) {
-        const uint32_t s = it % S, par = (it / S) & 1u;
+      for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
         if (!mbar_wait(done_bar(s), par, abort_flag)) { ok = false; break; }
         if (g + 1 == G.groups) {
           const StageHdr& h = hdrs[s];
@@ -397,9 +419,10 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   } else {
     // =============================== compute warps ===============================
     const uint32_t idx = threadIdx.x * kEpl;   // first element of this lane within the tile
-    uint32_t it = 0;
+    uint32_t s = 0, par = 0;
     bool ok = true;
     float acc[kEpl];
+    auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
       // PACKED: this warp's 128 elements lie in one small packet; the warp evaluates that packet's masks
       // itself, before it waits for the tile's data
@@ -435,8 +458,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           }
         }
       }
-      for (uint32_t g = 0; g < G.groups; ++g, ++it) {
-        const uint32_t s = it % S, par = (it / S) & 1u;
+      for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
         if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
         const StageHdr& h = hdrs[s];
         const uint64_t recv = PACKED ? my_recv : h.recv;
