@@ -102,7 +102,7 @@ constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * (sizeof(StageHdr)
 struct TmaPolicy {
   bool wide;      // 16 compute warps, one CTA per SM, 2048-element tiles (else 8 warps, two CTAs, 1024)
   int group;      // workers per pipeline stage: 4 or 8
-  bool early_stale;  // request the first stale replica copies before the tile's arithmetic (stages of 8 only)
+  int early_stale;   // stale copies: 0 = fetched in the drift phase, 16 = first ones requested before the tile's arithmetic, 1 = extra pipeline stages (stages of 8 only)
   uint32_t hints;
 };
 TmaPolicy tma_policy(const lossy_config& c) {
@@ -117,7 +117,10 @@ TmaPolicy tma_policy(const lossy_config& c) {
   t.hints = t.wide ? (pm >= 0.28 ? 3u : 0u) : ((c.W > 32 || pm >= 0.2) ? 3u : 0u);
   // early stale requests pay from about two stale replicas per tile at high loss: +8-10 % at W >= 16,
   // p = 0.3; at p = 0.1 they lose 1-2 % even with six stale replicas per tile (W = 64)
-  t.early_stale = t.group == 8 && (c.W - 1) * c.p_param >= 2.0 && c.p_param >= 0.15;
+  t.early_stale = t.group == 8 && (c.W - 1) * c.p_param >= 2.0 && c.p_param >= 0.15 ? 16 : 0;
+  // with dozens of stale replicas per tile their copies come as extra pipeline stages instead: +8 % at
+  // W = 64, p = 0.3, level at W = 32, a loss with fewer workers or lower loss (the extra stages cost depth)
+  if (t.early_stale && !t.wide && c.W >= 48 && c.p_param >= 0.2) t.early_stale = 1;
   return t;
 }
 
@@ -154,7 +157,8 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   G.groups = (c.W + kGroup - 1) / kGroup;
   uint32_t sb = G.grad_slots * kTile * gb + 3 * kTile * 4 + kTile * rb;
   G.stage_bytes = (sb + 127u) & ~127u;
-  const uint32_t budget = tma_smem_budget<CW>(ctx);
+  // behind the stages: fp64 drift sums per compute warp and replica (used by the stale-stage builds)
+  const uint32_t budget = tma_smem_budget<CW>(ctx) - CW * kMaxW * (uint32_t)sizeof(double);
   if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
   G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
   if (G.stages > (uint32_t)kMaxStages) G.stages = kMaxStages;
@@ -171,7 +175,7 @@ template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, boo
 int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
   auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS, PRE, PACKED>;
   constexpr int kThreadsTma = TmaShape<CW>::kThreads;
-  const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes;
+  const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes + CW * kMaxW * (uint32_t)sizeof(double);
   // launch bounds and the shared-memory budget guarantee kCtasPerSm resident CTAs per SM
   uint32_t blocks = (uint32_t)(ctx->num_sms * TmaShape<CW>::kCtasPerSm);
   if (blocks > G.num_tiles) blocks = G.num_tiles;
@@ -197,7 +201,9 @@ int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t
   const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
   const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
   if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
-  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
+  // stale copies as pipeline stages (PRE = 1) reuse the gradient slots: fp32 replicas with bf16 gradients do not fit
+  constexpr int PRE_WIDER = PRE == 1 ? 16 : PRE;
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE_WIDER, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE_WIDER, PACKED>(ctx, P, G, s, blocks);
   if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
   return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
 }
@@ -241,6 +247,7 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
     if (rc || *used) return rc;
   }
   return t.group == 4 ? try_tma<8, 4>(ctx, P, drift, s, blocks, used)
+         : t.early_stale == 1 ? try_tma<8, 8, 1>(ctx, P, drift, s, blocks, used)
          : t.early_stale ? try_tma<8, 8, 16>(ctx, P, drift, s, blocks, used)
                          : try_tma<8, 8>(ctx, P, drift, s, blocks, used);
 }

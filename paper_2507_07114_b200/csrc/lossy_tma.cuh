@@ -204,6 +204,10 @@ __device__ __forceinline__ void pack_bf16_lane(const float (&f)[kEpl], uint32_t 
 // arithmetic) so that its latency is hidden; 0 = every stale copy is fetched in the drift phase. The early
 // variant gains 8-10 % when a tile has several stale replicas (W >= 16 at p = 0.3) and costs 1-6 % when
 // it has about one or none, so both are built and the launch policy picks.
+// PRE = 1 selects another way altogether: the old copies of the replicas that miss a tile's broadcast come
+// through the pipeline as extra stages after the tile's last gradient group (up to GS copies per stage, in
+// the gradient slots), so the compute warps never wait on a global load. It needs replica elements no
+// larger than gradient elements and wins when a tile has many stale replicas.
 template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED = false>
 __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPerSm)
     lossy_fused_tma_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
@@ -212,6 +216,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   constexpr int kTile = TmaShape<CW>::kTile;
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
+  constexpr bool kStaleStages = DRIFTK && PRE == 1 && !PACKED;   // stale copies arrive as pipeline stages
+  static_assert(!kStaleStages || (sizeof(typename RT::raw) <= sizeof(typename GT::raw) && GS == 8), "stale stages reuse the gradient slots");
   // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) |
   //         stale masks per sub-packet of the PACKED build (kMaxStages x 64 B) | stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
@@ -220,6 +226,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   PackedStale* pks = reinterpret_cast<PackedStale*>(smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr));
   unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale));
   const uint32_t S = G.stages;
+  // stale-stage builds: fp64 drift sums per compute warp and replica, behind the stages
+  double* warp_acc = reinterpret_cast<double*>(stage0 + (size_t)S * G.stage_bytes);
   const uint32_t off_th = G.grad_slots * kTile * kGB;
   const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4, off_wire = off_v + kTile * 4;
 
@@ -230,6 +238,9 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   auto done_bar = [&](uint32_t s) { return smem_u32(&bars[kMaxStages + s]); };
   auto empty_bar = [&](uint32_t s) { return smem_u32(&bars[2 * kMaxStages + s]); };
 
+  if constexpr (kStaleStages) {
+    for (uint32_t q = threadIdx.x; q < (uint32_t)kConsumerWarps * kMaxW; q += blockDim.x) warp_acc[q] = 0.0;
+  }
   if (threadIdx.x == 0) {
     *abort_flag = 0u;
     for (uint32_t s = 0; s < S; ++s) {
@@ -325,7 +336,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               P.burst_out[(size_t)P.K + k] = pbad;
             }
           }
-          if constexpr (DRIFTK) {
+          if constexpr (DRIFTK && !kStaleStages) {
             for (uint32_t i = lane; i < W; i += 32)
               if ((stale >> i) & 1ull)
                 bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
@@ -357,6 +368,37 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             armed_mask |= 1u << s;
             armed_par = (armed_par & ~(1u << s)) | (par << s);
             if (++s == S) { s = 0; par ^= 1u; }
+          }
+          if constexpr (kStaleStages) {
+            // the old copies of the replicas that miss this broadcast, up to kGroup per extra stage; lane u
+            // fetches the u-th of them into gradient slot u
+            uint64_t sm = stale;
+            while (ok && sm) {
+              if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
+              uint64_t ids = 0;
+              int mine = -1;
+#pragma unroll
+              for (int u = 0; u < kGroup; ++u)
+                if (sm) {
+                  const int i = __ffsll((long long)sm) - 1;
+                  sm &= sm - 1;
+                  ids |= 1ull << i;
+                  if (lane == u) mine = i;
+                }
+              unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+              if (lane == 0) {
+                StageHdr& h = hdrs[s];
+                h.recv = ids; h.stale = 0; h.e0 = e0; h.k = k; h.len = len; h.cnt = (uint32_t)__popcll(ids); h.last = 2u;
+                mbar_arrive_expect_tx(full_bar(s), (uint32_t)__popcll(ids) * len * kRB);
+              }
+              __syncwarp();
+              if (mine >= 0)
+                bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
+                         reinterpret_cast<const typename RT::raw*>(P.replicas[mine]) + e0, len * kRB, full_bar(s), lh, pol);
+              armed_mask |= 1u << s;
+              armed_par = (armed_par & ~(1u << s)) | (par << s);
+              if (++s == S) { s = 0; par ^= 1u; }
+            }
           }
         }
       }
@@ -410,6 +452,18 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           }
           bulk_commit();
           bulk_wait_read0();          // shared memory of this stage may be overwritten after this
+          __syncwarp();
+          if (lane == 0) mbar_arrive(empty_bar(s));
+          if constexpr (kStaleStages) {
+            // the tile's stale stages carry nothing to store: hand each back once the compute warps are done
+            for (uint32_t n = ((uint32_t)__popcll(stale) + kGroup - 1) / kGroup; ok && n > 0; --n) {
+              next_stage();
+              if (!mbar_wait(done_bar(s), par, abort_flag)) { ok = false; break; }
+              __syncwarp();
+              if (lane == 0) mbar_arrive(empty_bar(s));
+            }
+          }
+          continue;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar(s));
@@ -494,7 +548,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         float wire[kEpl];
         // The first stale copies are requested now, so that their (L2) latency hides behind the arithmetic
         // below; they are used in the drift phase after this warp has handed the stage to the store warp.
-        constexpr int kPre = PRE / LaneWords<RT>::value;   // PRE = 16: 8 bf16 or 4 fp32 copies
+        constexpr int kPre = kStaleStages ? 0 : PRE / LaneWords<RT>::value;   // PRE = 16: 8 bf16 or 4 fp32 copies
         uint32_t pre_raw[kPre > 0 ? kPre : 1][4];
         int pre_id[kPre > 0 ? kPre : 1];
         uint64_t stale_rest = stale;
@@ -578,7 +632,44 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         if (lane == 0) mbar_arrive(done_bar(s));
 
         // ---- drift of the replicas that missed this broadcast ---------------------
-        if constexpr (DRIFTK) {
+        if constexpr (kStaleStages) {
+          // their old copies follow as stages of up to kGroup copies in the gradient slots
+          uint64_t sm = stale;
+          while (sm) {
+            next_stage();
+            if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
+            const uint64_t ids = hdrs[s].recv;
+            const unsigned char* sst = stage0 + (size_t)s * G.stage_bytes;
+            const uint32_t n_in = (uint32_t)__popcll(ids);
+            float sq[kGroup];
+#pragma unroll
+            for (int u = 0; u < kGroup; ++u) {
+              sq[u] = 0.0f;
+              if (active && (uint32_t)u < n_in) {
+                float old[kEpl];
+                lds_lane<RT>(sst + (size_t)u * kTile * kGB, idx, old);
+#pragma unroll
+                for (int x = 0; x < kEpl; ++x) {
+                  const float d = __fsub_rn(old[x], wire[x]);
+                  sq[u] = __fadd_rn(sq[u], __fmul_rn(d, d));
+                }
+              }
+            }
+            // all copies' warp totals at once; the first lane of segment u adds copy u's total to this warp's
+            // fp64 sum of that replica
+            const float tot = warp_sum_multi<kGroup>(sq, lane);
+            const uint32_t u = (uint32_t)lane / (32u / kGroup);
+            if ((lane & (32 / kGroup - 1)) == 0 && u < n_in) {
+              uint64_t t = ids;
+              for (uint32_t q = 0; q < u; ++q) t &= t - 1;
+              warp_acc[warp * kMaxW + (__ffsll((long long)t) - 1)] += (double)tot;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(done_bar(s));
+            sm &= ~ids;
+          }
+          if (!ok) break;
+        } else if constexpr (DRIFTK) {
 #pragma unroll
           for (int b = 0; b < kPre; ++b) {
             if (pre_id[b] >= 0) {
@@ -650,12 +741,14 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   __syncthreads();
   if (*abort_flag && threadIdx.x == 0) atomicExch(G.status, 1u);
   if constexpr (DRIFTK) {
-    double* sh = reinterpret_cast<double*>(stage0);   // stages are idle now
-    if (warp < kConsumerWarps) {
-      sh[warp * kMaxW + lane] = dacc0;
-      sh[warp * kMaxW + lane + 32] = dacc1;
+    double* sh = kStaleStages ? warp_acc : reinterpret_cast<double*>(stage0);   // stages are idle now
+    if constexpr (!kStaleStages) {
+      if (warp < kConsumerWarps) {
+        sh[warp * kMaxW + lane] = dacc0;
+        sh[warp * kMaxW + lane + 32] = dacc1;
+      }
+      __syncthreads();
     }
-    __syncthreads();
     if (threadIdx.x < kMaxW) {
       double t = 0.0;
 #pragma unroll

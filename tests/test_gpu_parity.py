@@ -86,6 +86,10 @@ EDGE = [
     ("bulk_w17_two_groups", 17, 2048 * 33, 2048, 0.3, "adam", "bf16", "bf16", SKIP),
     ("bulk_f32_everything", 9, 1024 * 55 + 1000, 1024, 0.1, "adam", "f32", "f32", LOSSLESS),
     ("bulk_fewer_tiles_than_ctas", 8, 4096 * 3, 4096, 0.3, "adam", "bf16", "bf16", 0),
+    # many workers at high loss: the stale replicas' old copies travel as extra pipeline stages
+    ("bulk_w64_stale_stages", 64, 1024 * 70 + 8, 1024, 0.3, "adam", "bf16", "bf16", 0),
+    ("bulk_w48_stale_stages_f32", 48, 2048 * 21, 2048, 0.25, "sgd", "f32", "f32", 0),
+    ("bulk_w50_stale_stages_mixed", 50, 1032 * 33 + 16, 1032, 0.45, "adam", "f32", "bf16", LOSSLESS),
     # small packets: a tile of the bulk-copy kernel packs several whole packets
     ("bulk_packed_256_w16_last_tile_short", 16, 256 * 37 + 100, 256, 0.2, "adam", "bf16", "bf16", 0),
     ("bulk_packed_128_w40", 40, 128 * 50 + 8, 128, 0.3, "sgd", "bf16", "bf16", 0),
