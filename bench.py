@@ -38,7 +38,7 @@ WORKLOAD = "cfg2_w8_layer_adam"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the fused kernel, from the ncu capture
-# of a small case of the same kernel (Nsight Compute, --set full): 1770.1 MB on a 33,554,432-element cut of the
+# of a small case of the same kernel (Nsight Compute, --set full): 1770.4 MB on a 33,554,432-element cut of the
 # workload, scaled by the elements processed (traffic is proportional to them).
 NCU_TRAFFIC_SMALL_CASE = (1770.4e6, 33554432)
 

@@ -58,10 +58,12 @@ enum {
   /* A packet that received nothing leaves theta, m, v untouched. Default: the
    * estimate is exactly 0 and is fed to the unmodified optimizer. */
   LOSSY_ZERO_SKIP = 2u,
-  /* lossy_fused_step always uses the register-path kernel. Default: complete packets go through
-   * the bulk-copy (TMA) pipeline when they hold at least 1024 elements, or when they are a
-   * multiple of 128 that divides the tile and the measured policy favours it (low loss, moderate
-   * worker count; that build also fetches the dropped packets of a tile). Same state either way. */
+  /* Every entry point uses the register-path kernel. Default: complete packets go through the
+   * bulk-copy (TMA) pipelines (one for the fused step, one per single-phase call) when they hold
+   * at least 1024 elements; the fused step also when they are a multiple of 128 that divides
+   * the tile and the measured policy favours it (few workers, or low loss; that build also
+   * fetches the dropped packets of a tile). Same parameters, replicas and masks either way; drift
+   * sums agree to rounding (another summation order). */
   LOSSY_REGISTER_PATH = 4u
 };
 
