@@ -77,6 +77,29 @@ def test_config2_full_layer_bucket():
     _run_full(w, steps=3, slab_packets=6, n_random=6, full_drift=True)
 
 
+def test_config2_full_layer_unfused_calls_match_the_fused_step():
+    """The four single-phase calls at full size, each on its own bulk-copy pipeline: the same masks,
+    parameters, moments, replicas and estimate as the fused step (itself checked against the oracle
+    above), bit for bit; drift norms to rounding (another summation order)."""
+    w = CFG["cfg2_w8_layer_adam"]
+    a, b = GpuRun(w), GpuRun(w)
+    for t in (1, 2):
+        gd = [workload.grad_slab(w, t, i, 0, w.n, "cuda") for i in range(w.W)]
+        a.step_fused(t, gd)
+        b.step_unfused(t, gd)
+        oa, ob = a.outputs(), b.outputs()
+        for key in ("count", "recv_bits", "stale_bits"):
+            assert_same(ob[key], oa[key], f"step {t} {key}")
+        assert torch.equal(a.ghat, b.ghat) and torch.equal(a.master, b.master)
+        assert torch.equal(a.m, b.m) and torch.equal(a.v, b.v)
+        for i in range(w.W):
+            assert torch.equal(a.replicas[i], b.replicas[i]), f"step {t} replica {i}"
+        assert_rel(ob["norms"], oa["norms"], f"step {t} norms", tol=2e-6)
+        del gd
+    L.lossy_device_status(a.ctx)
+    L.lossy_device_status(b.ctx)
+
+
 def test_config3_full_w64_sampled():
     w = CFG["cfg3_w64_layer_p10"]
     _run_full(w, steps=2, slab_packets=3, n_random=3, full_drift=False)

@@ -21,11 +21,11 @@ def test_config1_w4_sgd_fp32_all_steps(path_flag):
     run_parity(w, w.steps, flags=path_flag)
 
 
-@pytest.mark.parametrize("mode", ["bulk", "reg", "unfused"])
+@pytest.mark.parametrize("mode", ["bulk", "reg", "unfused", "unfused_reg"])
 def test_config2_shape_scaled_ragged(mode):
     # W=8, bf16 grads, Adam, P=2048: 37 packets + a short one whose length is not a multiple of 8
     w = workload.scaled(CFG["cfg2_w8_layer_adam"], 2048 * 37 + 1003)
-    run_parity(w, 12, fused=mode != "unfused", flags=REG if mode == "reg" else 0)
+    run_parity(w, 12, fused=not mode.startswith("unfused"), flags=REG if mode.endswith("reg") else 0)
 
 
 @PATHS
