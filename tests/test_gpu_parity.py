@@ -86,6 +86,8 @@ EDGE = [
     ("bulk_w17_two_groups", 17, 2048 * 33, 2048, 0.3, "adam", "bf16", "bf16", SKIP),
     ("bulk_f32_everything", 9, 1024 * 55 + 1000, 1024, 0.1, "adam", "f32", "f32", LOSSLESS),
     ("bulk_fewer_tiles_than_ctas", 8, 4096 * 3, 4096, 0.3, "adam", "bf16", "bf16", 0),
+    ("bulk_zero_skip_w2", 2, 1024 * 40 + 24, 1024, 0.6, "adam", "bf16", "bf16", SKIP),
+    ("bulk_zero_received_w3_f32", 3, 2048 * 25, 2048, 0.7, "sgd", "f32", "f32", 0),
     # many workers at high loss: the stale replicas' old copies travel as extra pipeline stages
     ("bulk_w64_stale_stages", 64, 1024 * 70 + 8, 1024, 0.3, "adam", "bf16", "bf16", 0),
     ("bulk_w48_stale_stages_f32", 48, 2048 * 21, 2048, 0.25, "sgd", "f32", "f32", 0),
@@ -110,7 +112,7 @@ def test_edge_cases(case, fused):
     name, W, n, P, p, opt, gd, rd, flags = case
     w = workload.Workload(name, W, n, P, p, opt, 1e-2 if opt == "sgd" else 3e-4, gd, rd, 5, seed=42)
     gpu, orc = run_parity(w, 5, fused=fused, flags=flags)
-    if name.startswith("heavy_loss"):
+    if name.startswith("heavy_loss") or name.startswith("bulk_zero"):
         assert int((gpu.count == 0).sum()) > 0          # the nothing-received fallback was exercised
 
 
