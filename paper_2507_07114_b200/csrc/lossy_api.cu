@@ -104,6 +104,8 @@ struct TmaPolicy {
   int group;      // workers per pipeline stage: 4 or 8
   int early_stale;   // stale copies: 0 = fetched in the drift phase, 16 = first ones requested before the tile's arithmetic, 1 = extra pipeline stages (stages of 8 only)
   uint32_t hints;
+  bool split;     // state slots apart from the stages (twin build, stages of 8, high loss)
+  uint32_t split_stages;
 };
 TmaPolicy tma_policy(const lossy_config& c) {
   const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
@@ -121,6 +123,13 @@ TmaPolicy tma_policy(const lossy_config& c) {
   // with dozens of stale replicas per tile their copies come as extra pipeline stages instead: +8 % at
   // W = 64, p = 0.3, level at W = 32, a loss with fewer workers or lower loss (the extra stages cost depth)
   if (t.early_stale && !t.wide && c.W >= 48 && c.p_param >= 0.2) t.early_stale = 1;
+  // State slots apart from the stages (one more gradient stage fits): the twin build at p >= 0.2, where the
+  // compute warps spend long on stale replicas and the extra stage keeps the loads going meanwhile: W = 32,
+  // p = 0.3: 0.89 -> 0.96; W = 48, p = 0.2: 0.91 -> 0.97; W = 64, p = 0.3: 0.90 -> 0.95. The fourth stage pays
+  // from about 6.5 stale replicas per tile; below that three (W = 24, p = 0.2: 0.93 -> 0.95), and at lower
+  // loss the plain build is as fast or faster (W = 64, p = 0.1: 0.96 against 0.94 with four stages).
+  t.split = !t.wide && t.group == 8 && c.W > 16 && c.p_param >= 0.2;
+  t.split_stages = (c.W - 1) * c.p_param >= 6.5 ? 4u : 3u;
   return t;
 }
 
@@ -134,7 +143,7 @@ uint32_t tma_smem_budget(const lossy_ctx* ctx) {
   return budget;
 }
 
-template <int CW, int GS, bool PACKED>
+template <int CW, int GS, bool PACKED, bool SPLIT>
 bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   constexpr uint32_t kGroup = GS;
   constexpr uint32_t kTile = TmaShape<CW>::kTile;
@@ -155,13 +164,17 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
   G.grad_slots = c.W < (uint32_t)kGroup ? c.W : (uint32_t)kGroup;
   G.groups = (c.W + kGroup - 1) / kGroup;
-  uint32_t sb = G.grad_slots * kTile * gb + 3 * kTile * 4 + kTile * rb;
+  const uint32_t state = 3 * kTile * 4 + kTile * rb;           // theta, m, v and the wire tile
+  const uint32_t sb = G.grad_slots * kTile * gb + (SPLIT ? 0u : state);
   G.stage_bytes = (sb + 127u) & ~127u;
-  // behind the stages: fp64 drift sums per compute warp and replica (used by the stale-stage builds)
-  const uint32_t budget = tma_smem_budget<CW>(ctx) - CW * kMaxW * (uint32_t)sizeof(double);
+  G.state_bytes = SPLIT ? (state + 127u) & ~127u : 0u;
+  // behind the stages: the two state slots of the SPLIT builds, and fp64 drift sums per compute warp and
+  // replica (used by the stale-stage builds)
+  const uint32_t budget = tma_smem_budget<CW>(ctx) - CW * kMaxW * (uint32_t)sizeof(double) - 2u * G.state_bytes;
   if (budget < kTmaSmemFixed + 2 * G.stage_bytes) return false;
   G.stages = (budget - kTmaSmemFixed) / G.stage_bytes;
-  if (G.stages > (uint32_t)kMaxStages) G.stages = kMaxStages;
+  const uint32_t cap = SPLIT ? tma_policy(c).split_stages : 4u;   // with the state in the stage a fifth measured no faster
+  if (G.stages > cap) G.stages = cap;
   // One tile per stage (a single worker group): with a fourth stage the loads run too far ahead of the
   // stores (W = 4, p = 0.1: 0.98 of the copy rate with three stages, 0.92 with four; W = 2: 0.96 / 0.95);
   // a single worker still gains from the fourth (0.97 / 0.91).
@@ -175,11 +188,11 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   return true;
 }
 
-template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED>
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED, bool SPLIT>
 int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS, PRE, PACKED>;
+  auto kern = lossy_fused_tma_kernel<GT, RT, OPT, DRIFTK, CW, GS, PRE, PACKED, SPLIT>;
   constexpr int kThreadsTma = TmaShape<CW>::kThreads;
-  const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes + CW * kMaxW * (uint32_t)sizeof(double);
+  const uint32_t smem = kTmaSmemFixed + G.stages * G.stage_bytes + 2u * G.state_bytes + CW * kMaxW * (uint32_t)sizeof(double);
   // launch bounds and the shared-memory budget guarantee kCtasPerSm resident CTAs per SM
   uint32_t blocks = (uint32_t)(ctx->num_sms * TmaShape<CW>::kCtasPerSm);
   if (blocks > G.num_tiles) blocks = G.num_tiles;
@@ -199,27 +212,27 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   return LOSSY_OK;
 }
 
-template <bool DRIFTK, int CW, int GS, int PRE, bool PACKED>
+template <bool DRIFTK, int CW, int GS, int PRE, bool PACKED, bool SPLIT>
 int dispatch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
   const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
   const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
   const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
-  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
+  if (gb && rb) return adam ? launch_tma<BF16, BF16, 1, DRIFTK, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks) : launch_tma<BF16, BF16, 0, DRIFTK, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks);
   // stale copies as pipeline stages (PRE = 1) reuse the gradient slots: fp32 replicas with bf16 gradients do not fit
   constexpr int PRE_WIDER = PRE == 1 ? 16 : PRE;
-  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE_WIDER, PACKED>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE_WIDER, PACKED>(ctx, P, G, s, blocks);
-  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
-  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_tma<BF16, F32, 1, DRIFTK, CW, GS, PRE_WIDER, PACKED, SPLIT>(ctx, P, G, s, blocks) : launch_tma<BF16, F32, 0, DRIFTK, CW, GS, PRE_WIDER, PACKED, SPLIT>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_tma<F32, BF16, 1, DRIFTK, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks) : launch_tma<F32, BF16, 0, DRIFTK, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks);
+  return adam ? launch_tma<F32, F32, 1, DRIFTK, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks) : launch_tma<F32, F32, 0, DRIFTK, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks);
 }
 
-template <int CW, int GS, int PRE = 0, bool PACKED = false>
+template <int CW, int GS, int PRE = 0, bool PACKED = false, bool SPLIT = false>
 int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
   TmaGeom G = {};
-  if (!tma_geometry<CW, GS, PACKED>(ctx, G)) return LOSSY_OK;
+  if (!tma_geometry<CW, GS, PACKED, SPLIT>(ctx, G)) return LOSSY_OK;
   *used = true;
   // without drift norms nothing reads the stale copies: the plain build serves
-  return drift ? dispatch_tma<true, CW, GS, PRE, PACKED>(ctx, P, G, s, blocks)
-               : dispatch_tma<false, CW, GS, 0, PACKED>(ctx, P, G, s, blocks);
+  return drift ? dispatch_tma<true, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks)
+               : dispatch_tma<false, CW, GS, 0, PACKED, SPLIT>(ctx, P, G, s, blocks);
 }
 
 // Run the build the policy picks; *used stays false when no bulk-copy launch fits (packets shorter
@@ -244,6 +257,12 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
       int rc = try_tma<8, 8, 0, true>(ctx, P, drift, s, blocks, used);
       if (rc || *used) return rc;
     }
+  }
+  if (t.split) {
+    // the state lives in its own two-slot ring (SPLIT builds, twin geometry only)
+    return t.early_stale == 1 ? try_tma<8, 8, 1, false, true>(ctx, P, drift, s, blocks, used)
+           : t.early_stale ? try_tma<8, 8, 16, false, true>(ctx, P, drift, s, blocks, used)
+                           : try_tma<8, 8, 0, false, true>(ctx, P, drift, s, blocks, used);
   }
   if (t.wide) {
     int rc = t.group == 4 ? try_tma<16, 4>(ctx, P, drift, s, blocks, used)

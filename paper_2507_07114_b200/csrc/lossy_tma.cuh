@@ -38,8 +38,8 @@ template <int CW> struct TmaShape {
 };
 constexpr int kStaleBatch = 4;                            // stale replica packets in flight per compute lane (8 measured slower)
 constexpr int kMaxStages = 4;                             // deeper pipelines measured no faster
-constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 x kMaxStages x 8 B) and the abort flag
-static_assert(3 * kMaxStages * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
+constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 per stage + 4 of the state slots, 8 B each) and the abort flag
+static_assert((3 * kMaxStages + 4) * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
 constexpr uint32_t kMaxPolls = 1u << 22;
 
 struct TmaGeom {
@@ -47,6 +47,7 @@ struct TmaGeom {
   uint32_t tiles_per_packet;
   uint32_t stages;
   uint32_t stage_bytes;       // per stage, 128-byte multiple
+  uint32_t state_bytes;       // SPLIT builds: one state slot (theta, m, v, wire tile), 128-byte multiple
   uint32_t groups;            // ceil(W / GS)
   uint32_t grad_slots;        // min(W, GS)
   uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores
@@ -208,7 +209,10 @@ __device__ __forceinline__ void pack_bf16_lane(const float (&f)[kEpl], uint32_t 
 // through the pipeline as extra stages after the tile's last gradient group (up to GS copies per stage, in
 // the gradient slots), so the compute warps never wait on a global load. It needs replica elements no
 // larger than gradient elements and wins when a tile has many stale replicas.
-template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED = false>
+// SPLIT: theta / m / v and the wire tile live in a ring of two state slots with barriers of their own
+// instead of in every stage, so that a stage is gradient slots only and more of them fit (a tile of W > 8
+// workers takes several stages, of which only the last needs the state).
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, int GS, int PRE, bool PACKED = false, bool SPLIT = false>
 __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPerSm)
     lossy_fused_tma_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
   constexpr int kConsumerWarps = CW;
@@ -217,6 +221,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
   constexpr bool kStaleStages = DRIFTK && PRE == 1 && !PACKED;   // stale copies arrive as pipeline stages
+  static_assert(!(SPLIT && PACKED), "the PACKED builds keep the state in the stage");
   static_assert(!kStaleStages || (sizeof(typename RT::raw) <= sizeof(typename GT::raw) && GS == 8), "stale stages reuse the gradient slots");
   // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) |
   //         stale masks per sub-packet of the PACKED build (kMaxStages x 64 B) | stages
@@ -226,9 +231,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   PackedStale* pks = reinterpret_cast<PackedStale*>(smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr));
   unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale));
   const uint32_t S = G.stages;
-  // stale-stage builds: fp64 drift sums per compute warp and replica, behind the stages
-  double* warp_acc = reinterpret_cast<double*>(stage0 + (size_t)S * G.stage_bytes);
-  const uint32_t off_th = G.grad_slots * kTile * kGB;
+  // SPLIT builds: two state slots behind the stages
+  unsigned char* state0 = stage0 + (size_t)S * G.stage_bytes;
+  // stale-stage builds: fp64 drift sums per compute warp and replica, behind everything else
+  double* warp_acc = reinterpret_cast<double*>(state0 + (SPLIT ? 2u * G.state_bytes : 0u));
+  const uint32_t off_th = SPLIT ? 0u : G.grad_slots * kTile * kGB;   // within the stage, or within the state slot
   const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4, off_wire = off_v + kTile * 4;
 
   const int lane = threadIdx.x & 31;
@@ -237,6 +244,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   auto full_bar = [&](uint32_t s) { return smem_u32(&bars[s]); };
   auto done_bar = [&](uint32_t s) { return smem_u32(&bars[kMaxStages + s]); };
   auto empty_bar = [&](uint32_t s) { return smem_u32(&bars[2 * kMaxStages + s]); };
+  auto sfull_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kMaxStages + q]); };        // SPLIT: state slot loaded
+  auto sempty_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kMaxStages + 2 + q]); };   // SPLIT: state slot stored
 
   if constexpr (kStaleStages) {
     for (uint32_t q = threadIdx.x; q < (uint32_t)kConsumerWarps * kMaxW; q += blockDim.x) warp_acc[q] = 0.0;
@@ -248,6 +257,12 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       mbar_init(done_bar(s), kConsumerWarps);
       mbar_init(empty_bar(s), 1);
     }
+    if constexpr (SPLIT) {
+      for (uint32_t q = 0; q < 2; ++q) {
+        mbar_init(sfull_bar(q), 1);
+        mbar_init(sempty_bar(q), 1);
+      }
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
   }
@@ -258,6 +273,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   if (warp == kConsumerWarps) {
     // =============================== producer warp ===============================
     uint32_t s = 0, par = 0, armed_mask = 0, armed_par = 0;
+    uint32_t sq = 0, spar = 0, sarmed_mask = 0, sarmed_par = 0;   // SPLIT: state slot ring
     bool ok = true;
     const bool lh = G.hints & 1u;
     const uint64_t pol = policy_evict_first();
@@ -342,14 +358,29 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
                 bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
           }
           if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
+          if constexpr (SPLIT) {
+            // the tile's theta / m / v go to state slot sq, ahead of its gradient groups
+            if (!mbar_wait(sempty_bar(sq), spar ^ 1u, abort_flag)) { ok = false; break; }
+            unsigned char* sb = state0 + (size_t)sq * G.state_bytes;
+            if (lane == 0) mbar_arrive_expect_tx(sfull_bar(sq), (OPT == 1 ? 3u : 1u) * len * 4u);
+            __syncwarp();
+            if (lane == 8) bulk_g2s(smem_u32(sb + off_th), P.master + e0, len * 4u, sfull_bar(sq), lh, pol);
+            if constexpr (OPT == 1) {
+              if (lane == 9) bulk_g2s(smem_u32(sb + off_m), P.m + e0, len * 4u, sfull_bar(sq), lh, pol);
+              if (lane == 10) bulk_g2s(smem_u32(sb + off_v), P.v + e0, len * 4u, sfull_bar(sq), lh, pol);
+            }
+            sarmed_mask |= 1u << sq;
+            sarmed_par = (sarmed_par & ~(1u << sq)) | (spar << sq);
+            if (++sq == 2u) { sq = 0; spar ^= 1u; }
+          }
           for (uint32_t g = 0; g < G.groups; ++g) {
             if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
-            const bool last = g + 1 == G.groups;
+            const bool last = !SPLIT && g + 1 == G.groups;   // the stage that also carries the state
             const uint32_t bits = (uint32_t)(recv >> (g * kGroup)) & ((1u << kGroup) - 1u);
             unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
             if (lane == 0) {
               StageHdr& h = hdrs[s];
-              h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
+              h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = g + 1 == G.groups ? 1u : 0u;
               uint32_t bytes = __popc(bits) * len * kGB;
               if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
               mbar_arrive_expect_tx(full_bar(s), bytes);
@@ -409,10 +440,16 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         if ((armed_mask >> q) & 1u)
           for (uint32_t i = 0; i < (1u << 16); ++i)
             if (mbar_try_wait(full_bar(q), (armed_par >> q) & 1u)) break;
+      if constexpr (SPLIT) {
+        for (uint32_t q = 0; q < 2; ++q)
+          if ((sarmed_mask >> q) & 1u)
+            for (uint32_t i = 0; i < (1u << 16); ++i)
+              if (mbar_try_wait(sfull_bar(q), (sarmed_par >> q) & 1u)) break;
+      }
     }
   } else if (warp == kConsumerWarps + 1) {
     // ================================ store warp =================================
-    uint32_t s = 0, par = 0;
+    uint32_t s = 0, par = 0, sq = 0;
     bool ok = true;
     const bool sh_hint = G.hints & 2u;
     const uint64_t pol = policy_evict_first();
@@ -424,7 +461,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           const StageHdr& h = hdrs[s];
           const uint64_t e0 = h.e0, stale = h.stale;
           const uint32_t len = h.len;
-          unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+          unsigned char* st = SPLIT ? state0 + (size_t)sq * G.state_bytes : stage0 + (size_t)s * G.stage_bytes;
           if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u, sh_hint, pol);
           if constexpr (OPT == 1) {
             if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u, sh_hint, pol);
@@ -454,6 +491,10 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           bulk_wait_read0();          // shared memory of this stage may be overwritten after this
           __syncwarp();
           if (lane == 0) mbar_arrive(empty_bar(s));
+          if constexpr (SPLIT) {
+            if (lane == 0) mbar_arrive(sempty_bar(sq));
+            sq ^= 1u;
+          }
           if constexpr (kStaleStages) {
             // the tile's stale stages carry nothing to store: hand each back once the compute warps are done
             for (uint32_t n = ((uint32_t)__popcll(stale) + kGroup - 1) / kGroup; ok && n > 0; --n) {
@@ -473,7 +514,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   } else {
     // =============================== compute warps ===============================
     const uint32_t idx = threadIdx.x * kEpl;   // first element of this lane within the tile
-    uint32_t s = 0, par = 0;
+    uint32_t s = 0, par = 0, sq = 0, spar = 0;
     bool ok = true;
     float acc[kEpl];
     auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
@@ -540,6 +581,12 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           continue;
         }
         // ---- last group of the tile: estimate, update, wire value -----------------
+        unsigned char* sb = st;       // where theta / m / v and the wire tile live
+        if constexpr (SPLIT) {
+          if (!mbar_wait(sfull_bar(sq), spar, abort_flag)) { ok = false; break; }
+          sb = state0 + (size_t)sq * G.state_bytes;
+          if (++sq == 2u) { sq = 0; spar ^= 1u; }
+        }
         const uint32_t cnt = PACKED ? (uint32_t)__popcll(my_recv) : h.cnt;
         const uint64_t stale = PACKED ? my_stale : h.stale, e0 = h.e0;
         if constexpr (PACKED) {
@@ -586,11 +633,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             store_words<kEpl>(P.ghat + e0 + idx, gw);
           }
           float th[kEpl], m[kEpl], v[kEpl];
-          lds_lane<F32>(st + off_th, idx, th);
+          lds_lane<F32>(sb + off_th, idx, th);
           if (!((P.flags & 2u) && cnt == 0)) {
             if constexpr (OPT == 1) {
-              lds_lane<F32>(st + off_m, idx, m);
-              lds_lane<F32>(st + off_v, idx, v);
+              lds_lane<F32>(sb + off_m, idx, m);
+              lds_lane<F32>(sb + off_v, idx, v);
             }
 #pragma unroll
             for (int x = 0; x < kEpl; ++x) {
@@ -607,20 +654,20 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
                 v[x] = vn;
               }
             }
-            sts_lane_f32(st + off_th, idx, th);
+            sts_lane_f32(sb + off_th, idx, th);
             if constexpr (OPT == 1) {
-              sts_lane_f32(st + off_m, idx, m);
-              sts_lane_f32(st + off_v, idx, v);
+              sts_lane_f32(sb + off_m, idx, m);
+              sts_lane_f32(sb + off_v, idx, v);
             }
           }
           if constexpr (RT::kVecs == 2) {
-            sts_lane_f32(st + off_wire, idx, th);
+            sts_lane_f32(sb + off_wire, idx, th);
 #pragma unroll
             for (int x = 0; x < kEpl; ++x) wire[x] = th[x];
           } else {
             uint32_t ww[4];
             pack_bf16_lane(th, ww);
-            store_words<kEpl / 2>(st + off_wire + (size_t)idx * 2, ww);
+            store_words<kEpl / 2>(sb + off_wire + (size_t)idx * 2, ww);
             unpack_lane<BF16>(ww, wire);
           }
         } else {
