@@ -120,9 +120,6 @@ TmaPolicy tma_policy(const lossy_config& c) {
   // early stale requests pay from about two stale replicas per tile at high loss: +8-10 % at W >= 16,
   // p = 0.3; at p = 0.1 they lose 1-2 % even with six stale replicas per tile (W = 64)
   t.early_stale = t.group == 8 && (c.W - 1) * c.p_param >= 2.0 && c.p_param >= 0.15 ? 16 : 0;
-  // with dozens of stale replicas per tile their copies come as extra pipeline stages instead: +8 % at
-  // W = 64, p = 0.3, level at W = 32, a loss with fewer workers or lower loss (the extra stages cost depth)
-  if (t.early_stale && !t.wide && c.W >= 48 && c.p_param >= 0.2) t.early_stale = 1;
   // State slots apart from the stages (one more gradient stage fits): the twin build at p >= 0.2, where the
   // compute warps spend long on stale replicas and the extra stage keeps the loads going meanwhile: W = 32,
   // p = 0.3: 0.89 -> 0.96; W = 48, p = 0.2: 0.91 -> 0.97; W = 64, p = 0.3: 0.90 -> 0.95. The fourth stage pays
@@ -130,6 +127,11 @@ TmaPolicy tma_policy(const lossy_config& c) {
   // loss the plain build is as fast or faster (W = 64, p = 0.1: 0.96 against 0.94 with four stages).
   t.split = !t.wide && t.group == 8 && c.W > 16 && c.p_param >= 0.2;
   t.split_stages = (c.W - 1) * c.p_param >= 6.5 ? 4u : 3u;
+  // With the fourth stage the stale replicas' old copies come through the pipeline as extra stages instead
+  // of being read by the compute warps (W = 64, p = 0.3: 0.88 -> 0.95; W = 48, p = 0.3: 0.91 -> 0.97; W = 17,
+  // p = 0.5: 0.71 -> 0.79); with fewer stale replicas per tile the early requests stay ahead (W = 24, p = 0.2:
+  // 0.95 against 0.92).
+  if (t.split && t.split_stages == 4u) t.early_stale = 1;
   return t;
 }
 
@@ -271,7 +273,6 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
     if (rc || *used) return rc;
   }
   return t.group == 4 ? try_tma<8, 4>(ctx, P, drift, s, blocks, used)
-         : t.early_stale == 1 ? try_tma<8, 8, 1>(ctx, P, drift, s, blocks, used)
          : t.early_stale ? try_tma<8, 8, 16>(ctx, P, drift, s, blocks, used)
                          : try_tma<8, 8>(ctx, P, drift, s, blocks, used);
 }
