@@ -3,9 +3,9 @@
 // One CTA = CW compute warps + 1 producer warp + 1 store warp (see TmaShape for the two builds).
 // The bucket's full packets are cut into tiles of at most kTile contiguous elements inside one
 // packet (kTile = 128 * CW), so one set of delivery masks covers a tile. Per tile and per group of
-// up to GS (4 or 8) workers the producer arms an mbarrier and issues 1-D bulk copies global -> shared memory for the
-// DELIVERED workers' pieces only (dropped packets are never read) and, with the last group, for
-// theta / m / v. Compute warps sum the pieces in ascending worker order from shared memory,
+// up to GS (4 or 8) workers the producer arms an mbarrier and issues 1-D bulk copies global ->
+// shared memory for the DELIVERED workers' pieces only (dropped packets are never read) and, with
+// the last group, for theta / m / v. Compute warps sum the pieces in ascending worker order from shared memory,
 // divide by the received count, run the optimizer in place in shared memory and write the wire
 // value (fp32 or RNE bf16) once; the store warp then fans that single shared-memory tile out with
 // one bulk copy per replica that receives the broadcast, plus theta / m / v. Replicas that miss
@@ -14,8 +14,11 @@
 //
 // Template variants, picked per context by the host's launch policy: CW (compute warps: 16 = one CTA per
 // SM with 2048-element tiles, 8 = two CTAs per SM with 1024-element tiles), GS (workers per pipeline stage, 4
-// or 8), PRE (registers per lane for stale replica data requested before the tile's arithmetic, 0 or 16) and
-// PACKED (packets shorter than a tile: several whole packets per tile, masks evaluated by the compute warps).
+// or 8), PRE (how the old copies of stale replicas are read: 0 = by the compute warps in the drift phase, 16 =
+// the first ones requested before the tile's arithmetic into 16 registers per lane, 1 = as extra pipeline
+// stages), PACKED (packets shorter than a tile: several whole packets per tile, masks evaluated by the
+// compute warps) and SPLIT (theta / m / v and the wire tile in two state slots of their own, stages of
+// gradient slots only).
 // Drift norms are finalised by the last CTA to finish (fence + ticket counter; nothing waits on another CTA).
 //
 // Every wait on an mbarrier is bounded: after kMaxPolls unsuccessful polls the CTA raises a
