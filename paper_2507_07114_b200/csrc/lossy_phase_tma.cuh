@@ -16,7 +16,7 @@
 
 namespace lossy {
 
-constexpr int kPhaseMaxStages = 8;     // read-mostly phases gain from every stage that fits
+constexpr int kPhaseMaxStages = 8;     // as many as fit, up to eight (the host caps the optimizer step at three)
 static_assert(3 * kPhaseMaxStages * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
 
 // bytes of one pipeline stage; `slots` = arrays of the streamed group (AGG, DRIFT), `eb` = their element size
