@@ -235,6 +235,7 @@ def main():
                        grad_dtype=gdt, replica_dtype=rdt, optimizer=w.optimizer, lr=w.lr, beta1=w.beta1,
                        beta2=w.beta2, eps=w.eps, packet_base=w.packet_base,
                        flags=L.LOSSY_REGISTER_PATH if args.register_path else 0, **rng_kw)
+    plan = L.lossy_describe_plan(ctx, True)       # the build the library's launch policy picks for this workload
     master = workload.theta0_slab(w, e_off, e_off + w.n, dev)
     m = torch.zeros_like(master) if adam else None
     v = torch.zeros_like(master) if adam else None
@@ -348,8 +349,8 @@ def main():
                          "traffic": (NCU_TRAFFIC_SMALL_CASE[0] * w.n / NCU_TRAFFIC_SMALL_CASE[1]
                                      if pristine else None),
                          "peak_source": peak_src + " (MEASURED_PEAKS.json hbm_gbs)" if peak_src == "measured"
-                         else peak_src, "kernel": ("lossy_kernel<AGG|STEP|BCAST|DRIFT>" if args.register_path else "lossy_fused_tma_kernel")
-                         + " (drift norms finalised by its last block)",
+                         else peak_src, "kernel": ("lossy_kernel<AGG|STEP|BCAST|DRIFT>" if plan.startswith("register") else "lossy_fused_tma_kernel")
+                         + " (drift norms finalised by its last block)", "build": plan,
                          "avg_launch_ms": avg_launch_ms, "min_launch_ms": min(per_launch_ms)},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
         }

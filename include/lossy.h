@@ -38,6 +38,7 @@
 #ifndef LOSSY_H_
 #define LOSSY_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -382,6 +383,15 @@ uint64_t lossy_num_packets(const lossy_ctx* ctx);
 
 /* lossy_kernel_launches — kernels this context has launched so far (0 for NULL). */
 uint64_t lossy_kernel_launches(const lossy_ctx* ctx);
+
+/* lossy_describe_plan — which kernel build lossy_fused_step would launch for the complete packets of
+ * this context, as text for logs and benchmarks: "bulk-copy wide|twin group=4|8 stale=late|early|staged
+ * [packed] [split] stages=N", or "register kernel" when no bulk-copy build fits (a ragged last packet goes
+ * to the register kernel in either case). with_drift != 0 asks for the call that also returns drift norms.
+ * Host only: launches nothing and allocates nothing. Writes at most size bytes including the terminator
+ * (truncating); buf is a host buffer owned by the caller. LOSSY_EINVAL for a NULL argument or size 0.
+ * The paper has no counterpart: the build choice is this library's measured launch policy. */
+int lossy_describe_plan(lossy_ctx* ctx, int with_drift, char* buf, size_t size);
 
 #ifdef __cplusplus
 }

@@ -23,6 +23,7 @@ EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_set_reliable", "lossy_packet_sqnorms", "lossy_aggregate", "lossy_step", "lossy_broadcast",
     "drift_norms", "drift_pairwise", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
+    "lossy_describe_plan",
 ]
 
 
@@ -104,6 +105,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_num_packets.argtypes = [vp]
     lib.lossy_kernel_launches.restype = u64
     lib.lossy_kernel_launches.argtypes = [vp]
+    lib.lossy_describe_plan.restype = C.c_int
+    lib.lossy_describe_plan.argtypes = [vp, C.c_int, C.c_char_p, C.c_size_t]
     if path == _build.LIB_PATH:
         _lib = lib
     return lib
@@ -268,3 +271,10 @@ def lossy_num_packets(ctx) -> int:
 
 def lossy_kernel_launches(ctx) -> int:
     return load_library().lossy_kernel_launches(ctx)
+
+
+def lossy_describe_plan(ctx, with_drift: bool = True) -> str:
+    """Text naming the kernel build lossy_fused_step would launch for this context's complete packets."""
+    buf = C.create_string_buffer(128)
+    _check(ctx, load_library().lossy_describe_plan(ctx, int(with_drift), buf, len(buf)))
+    return buf.value.decode()

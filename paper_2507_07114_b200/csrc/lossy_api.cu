@@ -31,6 +31,8 @@ struct lossy_ctx {
   uint32_t Tenter, Tstay;
   int smem_optin;        // largest dynamic shared memory a block may opt in to
   uint64_t launches;
+  char* plan;            // lossy_describe_plan: where try_tma notes the build it would launch (else NULL)
+  size_t plan_size;
   char err[256];
 };
 
@@ -232,6 +234,13 @@ int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   TmaGeom G = {};
   if (!tma_geometry<CW, GS, PACKED, SPLIT>(ctx, G)) return LOSSY_OK;
   *used = true;
+  if (ctx->plan) {
+    // dispatch_tma runs the early-request build where staged copies do not fit the gradient slots
+    const bool fits = !(ctx->cfg.grad_dtype == LOSSY_BF16 && ctx->cfg.replica_dtype == LOSSY_F32);
+    snprintf(ctx->plan, ctx->plan_size, "bulk-copy %s group=%d stale=%s%s%s stages=%u", CW == 16 ? "wide" : "twin", GS,
+             !drift || PRE == 0 ? "late" : PRE == 1 && fits ? "staged" : "early", PACKED ? " packed" : "",
+             SPLIT ? " split" : "", G.stages);
+  }
   // without drift norms nothing reads the stale copies: the plain build serves
   return drift ? dispatch_tma<true, CW, GS, PRE, PACKED, SPLIT>(ctx, P, G, s, blocks)
                : dispatch_tma<false, CW, GS, 0, PACKED, SPLIT>(ctx, P, G, s, blocks);
@@ -866,5 +875,22 @@ int lossy_mask_grid(lossy_ctx* ctx, uint64_t step, const uint32_t* src, const ui
 const char* lossy_last_error(const lossy_ctx* ctx) { return ctx ? ctx->err : "NULL context"; }
 uint64_t lossy_num_packets(const lossy_ctx* ctx) { return ctx ? ctx->K : 0; }
 uint64_t lossy_kernel_launches(const lossy_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int lossy_describe_plan(lossy_ctx* ctx, int with_drift, char* buf, size_t size) {
+  if (!ctx || !buf || size == 0) return LOSSY_EINVAL;
+  snprintf(buf, size, "register kernel");
+  if (ctx->cfg.n == 0) return LOSSY_OK;
+  Params P;
+  fill_common(ctx, 1, P);
+  uint32_t blocks = 0;
+  bool used = false;
+  ctx->plan = buf;
+  ctx->plan_size = size;
+  ctx->plan_only = true;             // sizes grids, launches nothing
+  const int rc = run_tma(ctx, P, with_drift != 0, nullptr, &blocks, &used);
+  ctx->plan_only = false;
+  ctx->plan = nullptr;
+  return rc;
+}
 
 }  // extern "C"

@@ -303,3 +303,30 @@ def test_host_gradient_entry_point_zero_copy_and_staged_match_the_device_path():
     with pytest.raises(L.LossyError):                      # pageable memory without staging buffers
         L.lossy_fused_step_host(paged.ctx, 5, gs, None, paged.master, paged.m, paged.v, paged.replicas, paged.norms,
                                 host_norms)
+
+
+def test_launch_policy_picks_the_expected_build_for_the_benchmark_configurations():
+    """lossy_describe_plan names the kernel build the fused step launches; the choices below are the
+    measured policy for the benchmark's configurations and for its corner cases."""
+    def plan(W, P, p, n=None, gd="bf16", rd="bf16", flags=0):
+        n = P * 4000 if n is None else n
+        ctx = L.lossy_init(W=W, n=n, packet_elems=P, p_grad=p, p_param=p, seed=1, grad_dtype=torch.bfloat16 if gd == "bf16" else torch.float32,
+                           replica_dtype=torch.bfloat16 if rd == "bf16" else torch.float32, optimizer="adam", lr=1e-3, flags=flags)
+        try:
+            return L.lossy_describe_plan(ctx, True), L.lossy_describe_plan(ctx, False)
+        finally:
+            L.lossy_destroy(ctx)
+
+    assert plan(8, 2048, 0.1)[0] == "bulk-copy wide group=4 stale=late stages=4"          # config 2
+    assert plan(64, 4096, 0.1)[0] == "bulk-copy twin group=8 stale=late stages=3"         # config 3
+    assert plan(4, 1024, 0.1, gd="f32", rd="f32")[0].startswith("bulk-copy twin group=4")  # config 1
+    assert plan(16, 1024, 0.3)[0] == "bulk-copy twin group=8 stale=early stages=3"        # config 5, P = 1024
+    assert plan(16, 256, 0.1)[0].startswith("bulk-copy wide group=8 stale=late packed")   # config 5, small packets, low loss
+    assert plan(16, 256, 0.3)[0] == "register kernel"                                     # ... and at high loss
+    assert plan(64, 4096, 0.3)[0] == "bulk-copy twin group=8 stale=staged split stages=4"
+    assert plan(24, 2048, 0.2)[0] == "bulk-copy twin group=8 stale=early split stages=3"
+    # fp32 replicas do not fit bf16 gradient slots: early requests instead of staged copies
+    assert plan(64, 4096, 0.3, rd="f32")[0] == "bulk-copy twin group=8 stale=early split stages=4"
+    assert plan(64, 4096, 0.3)[1] == "bulk-copy twin group=8 stale=late split stages=4"   # no drift norms asked for
+    assert plan(8, 2048, 0.1, flags=L.LOSSY_REGISTER_PATH)[0] == "register kernel"
+    assert plan(8, 2048, 0.1, n=1000)[0] == "register kernel"                             # no complete packet
