@@ -94,11 +94,12 @@ def run_point(w, steps, warmup=3, grad_sets=2, alg1=False, graph=False):
         torch.cuda.synchronize()
         graph_sps = reps * steps / (e0.elapsed_time(e1) * 1e-3)
         L.lossy_device_status(ctx)
+    plan = L.lossy_describe_plan(ctx, True)
     L.lossy_destroy(ctx)
     gbs = algorithmic_bytes(w, alg1) / (ms * 1e-3) / 1e9
     return {"workload": w.name + ("[alg1]" if alg1 else ""), "W": w.W, "P": w.packet_elems, "p": w.p, "ms_per_step": ms, "GBps": gbs,
             "frac_of_measured_peak": gbs / _peak(), "steps_per_s": 1e3 / ms, "max_drift_norm": float(worst.max()),
-            **({"steps_per_s_cuda_graph": graph_sps} if graph_sps else {})}
+            "build": plan, **({"steps_per_s_cuda_graph": graph_sps} if graph_sps else {})}
 
 
 def run_unfused(w, steps=20, warmup=3):
