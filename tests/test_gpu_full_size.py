@@ -105,6 +105,13 @@ def test_config3_full_w64_sampled():
     _run_full(w, steps=2, slab_packets=3, n_random=3, full_drift=False)
 
 
+def test_w64_high_loss_full_size_split_build_with_staged_stale_copies():
+    # W = 64 at p = 0.3: state slots apart from the stages, stale replicas' old copies as pipeline stages
+    w = workload.scaled(CFG["cfg3_w64_layer_p10"], workload.LAYER_ELEMS, p=0.3)
+    gpu = _run_full(w, steps=2, slab_packets=3, n_random=3, full_drift=False)
+    assert L.lossy_describe_plan(gpu.ctx) == "bulk-copy twin group=8 stale=staged split stages=4"
+
+
 def test_config5_point_full_size_small_packets_register_path():
     # P=256 takes the register-path kernel at full size
     w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.3)
