@@ -118,6 +118,13 @@ def test_config5_point_full_size_small_packets_register_path():
     _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
 
 
+def test_config5_point_full_size_small_packets_packed_build():
+    # P=256 at low loss takes the PACKED bulk-copy build (eight whole packets per tile) at full size
+    w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.05)
+    gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
+    assert L.lossy_describe_plan(gpu.ctx).startswith("bulk-copy wide group=8 stale=late packed")
+
+
 def test_drift_is_order_one_and_matches_the_stationary_constant_at_scale():
     """Bounded Model Drift at scale, as a property that holds at any size: with SGD and gradients
     redrawn i.i.d. every step, a replica's squared distance from the owners' values settles at
