@@ -117,8 +117,9 @@ TmaPolicy tma_policy(const lossy_config& c) {
   // stages of 4 workers (finer-grained pipeline) win for few workers at low loss: +5 % at W = 8, p = 0.1,
   // but -9 % at W = 8, p = 0.3; the crossover at W = 8 sits near p = 0.17
   t.group = c.W <= 4 ? 4 : (c.W <= 8 && pm < 0.175 ? 4 : 8);
-  // hints: +3-4 % on the twin build at W = 64 or at high loss, neutral to -2 % elsewhere
-  t.hints = t.wide ? (pm >= 0.28 ? 3u : 0u) : ((c.W > 32 || pm >= 0.2) ? 3u : 0u);
+  // hints: +2-4 % on the twin build at high loss, or at W = 64 from moderate loss (p = 0.1: 0.957 against
+  // 0.934); neutral to -2 % elsewhere (W = 64, p = 0.01: 0.944 against 0.961)
+  t.hints = t.wide ? (pm >= 0.28 ? 3u : 0u) : ((pm >= 0.2 || (c.W > 32 && pm >= 0.05)) ? 3u : 0u);
   // early stale requests pay from about two stale replicas per tile at high loss: +8-10 % at W >= 16,
   // p = 0.3; at p = 0.1 they lose 1-2 % even with six stale replicas per tile (W = 64)
   t.early_stale = t.group == 8 && (c.W - 1) * c.p_param >= 2.0 && c.p_param >= 0.15 ? 16 : 0;
