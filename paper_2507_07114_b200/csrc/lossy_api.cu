@@ -253,6 +253,18 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   *used = false;
   if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
   const TmaPolicy t = tma_policy(ctx->cfg);
+  {
+    // Packets of exactly half a wide tile with 13..16 workers at low loss: the PACKED wide build (two packets
+    // per tile, one CTA per SM) beats the twin build, whose pieces are 2 KB (W = 16: 0.96-0.98 against 0.93 up
+    // to p = 0.1; W = 13-14: 0.97-1.0 against 0.94 up to p = 0.05); beyond that its fetches of dropped packets
+    // cost more than the wider tile gains, and from 12 workers down the twin build is ahead at every p.
+    const lossy_config& c = ctx->cfg;
+    const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
+    if (c.packet_elems * 2u == (uint32_t)TmaShape<16>::kTile && c.W >= 13 && c.W <= 16 && pm <= (c.W == 16 ? 0.1 : 0.05)) {
+      int rc = try_tma<16, 8, 0, true>(ctx, P, drift, s, blocks, used);
+      if (rc || *used) return rc;
+    }
+  }
   if (ctx->cfg.packet_elems < (uint32_t)TmaShape<8>::kTile) {
     // Packets shorter than a tile: the PACKED builds, where they beat the register kernel. They fetch the
     // dropped sub-packets too, so they win at low loss (+8..17 % at W = 8-16, P = 256-512, p <= 0.1) and lose

@@ -322,6 +322,7 @@ def test_launch_policy_picks_the_expected_build_for_the_benchmark_configurations
     assert plan(4, 1024, 0.1, gd="f32", rd="f32")[0].startswith("bulk-copy twin group=4")  # config 1
     assert plan(16, 1024, 0.3)[0] == "bulk-copy twin group=8 stale=early stages=3"        # config 5, P = 1024
     assert plan(16, 256, 0.1)[0].startswith("bulk-copy wide group=8 stale=late packed")   # config 5, small packets, low loss
+    assert plan(16, 1024, 0.05)[0].startswith("bulk-copy wide group=8 stale=late packed")  # config 5, P = 1024, low loss: two packets per wide tile
     assert plan(16, 256, 0.3)[0] == "register kernel"                                     # ... and at high loss
     assert plan(64, 4096, 0.3)[0] == "bulk-copy twin group=8 stale=staged split stages=4"
     assert plan(24, 2048, 0.2)[0] == "bulk-copy twin group=8 stale=early split stages=3"
