@@ -33,6 +33,8 @@ CASES = [
     # name, W, n, P, p, opt, gd, rd, flags
     ("wide_ragged", 8, 2048 * 19 + 1003, 2048, 0.2, "adam", "bf16", "bf16", 0),
     ("twin_w40_short_last_tile", 40, 1032 * 23 + 512, 1032, 0.2, "adam", "bf16", "f32", 0),
+    ("twin_w64_split_staged", 64, 1024 * 30 + 16, 1024, 0.3, "adam", "bf16", "bf16", 0),
+    ("packed_1024_two_per_wide_tile", 16, 1024 * 21 + 8, 1024, 0.05, "adam", "bf16", "bf16", 0),
     ("packed_256", 16, 256 * 45 + 40, 256, 0.1, "adam", "bf16", "bf16", 0),
     ("packed_128_twin", 30, 128 * 77 + 8, 128, 0.1, "sgd", "f32", "bf16", 0),
     ("register_path", 8, 2048 * 7 + 5, 2048, 0.3, "adam", "bf16", "bf16", L.LOSSY_REGISTER_PATH),
