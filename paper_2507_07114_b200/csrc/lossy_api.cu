@@ -96,7 +96,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 }
 
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
-constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale));
+constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)) + 2 * sizeof(PackedMasks);
 
 // Launch policy of the bulk-copy pipeline, from sweeps on B200 over W = 2..64, p = 0.05..0.3
 // (CUDA-event timings of bench.py with each build forced): which of the four builds runs and whether its bulk copies carry an
@@ -183,7 +183,7 @@ bool tma_geometry(const lossy_ctx* ctx, TmaGeom& G) {
   // One tile per stage (a single worker group): with a fourth stage the loads run too far ahead of the
   // stores (W = 4, p = 0.1: 0.98 of the copy rate with three stages, 0.92 with four; W = 2: 0.96 / 0.95);
   // a single worker still gains from the fourth (0.97 / 0.91).
-  if (!PACKED && G.groups == 1 && c.W >= 2 && G.stages > 3u) G.stages = 3u;
+  if (G.groups == 1 && c.W >= 2 && G.stages > 3u) G.stages = 3u;
   G.tiles_per_packet = PACKED ? 1u : (c.packet_elems + kTile - 1) / kTile;
   const uint64_t tiles = PACKED ? (kfull + G.packets_per_tile - 1) / G.packets_per_tile : kfull * G.tiles_per_packet;
   if (tiles >= (1ull << 31)) return false;

@@ -41,8 +41,8 @@ template <int CW> struct TmaShape {
 };
 constexpr int kStaleBatch = 4;                            // stale replica packets in flight per compute lane (8 measured slower)
 constexpr int kMaxStages = 4;                             // deeper pipelines measured no faster
-constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 per stage + 4 of the state slots, 8 B each) and the abort flag
-static_assert((3 * kMaxStages + 4) * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
+constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 per stage, 4 of the state slots, 2 of the PACKED masks; 8 B each) and the abort flag
+static_assert((3 * kMaxStages + 6) * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
 constexpr uint32_t kMaxPolls = 1u << 22;
 
 struct TmaGeom {
@@ -67,6 +67,7 @@ struct TmaGeom {
 // sub-packets whose broadcast it received.
 constexpr int kMaxSub = 8;
 struct __align__(16) PackedStale { uint64_t stale[kMaxSub]; };
+struct __align__(16) PackedMasks { uint64_t recv[kMaxSub], stale[kMaxSub]; };   // a tile's masks, shared by its compute warps
 
 struct __align__(16) StageHdr {
   uint64_t recv, stale, e0;
@@ -227,12 +228,14 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   static_assert(!(SPLIT && PACKED), "the PACKED builds keep the state in the stage");
   static_assert(!kStaleStages || (sizeof(typename RT::raw) <= sizeof(typename GT::raw) && GS == 8), "stale stages reuse the gradient slots");
   // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) |
-  //         stale masks per sub-packet of the PACKED build (kMaxStages x 64 B) | stages
+  //         stale masks per sub-packet of the PACKED build (kMaxStages x 64 B) | two tiles' masks of the PACKED
+  //         build (2 x 128 B) | stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kTmaBarBytes - 4);
   StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + kTmaBarBytes);
   PackedStale* pks = reinterpret_cast<PackedStale*>(smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr));
-  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale));
+  PackedMasks* tmasks = reinterpret_cast<PackedMasks*>(smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)));   // [2]
+  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)) + 2 * sizeof(PackedMasks);
   const uint32_t S = G.stages;
   // SPLIT builds: two state slots behind the stages
   unsigned char* state0 = stage0 + (size_t)S * G.stage_bytes;
@@ -249,6 +252,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   auto empty_bar = [&](uint32_t s) { return smem_u32(&bars[2 * kMaxStages + s]); };
   auto sfull_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kMaxStages + q]); };        // SPLIT: state slot loaded
   auto sempty_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kMaxStages + 2 + q]); };   // SPLIT: state slot stored
+  auto mask_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kMaxStages + 4 + q]); };     // PACKED: a tile's masks are written
 
   if constexpr (kStaleStages) {
     for (uint32_t q = threadIdx.x; q < (uint32_t)kConsumerWarps * kMaxW; q += blockDim.x) warp_acc[q] = 0.0;
@@ -265,6 +269,9 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         mbar_init(sfull_bar(q), 1);
         mbar_init(sempty_bar(q), 1);
       }
+    }
+    if constexpr (PACKED) {
+      for (uint32_t q = 0; q < 2; ++q) mbar_init(mask_bar(q), kConsumerWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -521,31 +528,75 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     bool ok = true;
     float acc[kEpl];
     auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
+    // PACKED: this warp's 128 elements lie in one sub-packet of the tile, always the same one
+    const uint32_t my_sp = PACKED ? min((uint32_t)(threadIdx.x & ~31) * kEpl / P.P, (uint32_t)kMaxSub - 1u) : 0u;
+    uint32_t mbuf = 0, mpar = 0;                 // PACKED: buffer and phase of the shared tile masks
+    uint32_t pk_Wp = 32;
+    const bool pk_batched = PACKED && W <= 32 && !P.ghat_prev;
+    if (pk_batched) { pk_Wp = 1; while (pk_Wp < W) pk_Wp <<= 1; }
+    const uint32_t pk_lgWp = 31u - (uint32_t)__clz((int)pk_Wp);
+    // sub-packets per pass of draws: at most two, so that the work spreads over several warps instead of
+    // lengthening one warp's tile (with W <= 4 a single pass could cover all eight, and did so at a loss)
+    const uint32_t pk_Bp = min(32u >> pk_lgWp, 2u);
+    const uint32_t pk_wmask = pk_Wp == 32 ? 0xFFFFFFFFu : ((1u << pk_Wp) - 1u);
+    // PACKED: a tile's masks are evaluated once, one tile ahead, and shared through two alternating buffers
+    // (a warp that is ahead never overwrites masks still being read): with W <= 32 (not Algorithm 1) warp w
+    // takes the w-th batch of 32 / Wp sub-packets in one pass of draws; otherwise the first warp of each
+    // sub-packet takes its own. Every compute warp arrives on the buffer's barrier once per tile.
+    auto eval_masks = [&](uint32_t tile, uint32_t buf) {
+      const uint32_t kfirst = tile * G.packets_per_tile;
+      const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
+      const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;
+      PackedMasks& tm = tmasks[buf];
+      auto report = [&](uint32_t sp, uint64_t r, uint64_t st, uint64_t gbad, uint64_t pbad) {   // one lane
+        const uint32_t k = kfirst + sp;
+        tm.recv[sp] = r;
+        tm.stale[sp] = st;
+        if (P.count) P.count[k] = (uint8_t)__popcll(r);
+        if (P.recv_bits) P.recv_bits[k] = r;
+        if (P.stale_bits) P.stale_bits[k] = st;
+        if (P.burst_out) {
+          P.burst_out[k] = gbad;
+          P.burst_out[(size_t)P.K + k] = pbad;
+        }
+      };
+      if (pk_batched) {
+        const uint32_t q0 = (uint32_t)warp * pk_Bp;
+        if (q0 < npk) {
+          const uint32_t sp_l = q0 + ((uint32_t)lane >> pk_lgWp), i_l = (uint32_t)lane & (pk_Wp - 1u);
+          const uint32_t k_l = kfirst + (sp_l < npk ? sp_l : 0u);
+          const BatchDraws d = batch_draws<AGG | BCAST>(P, k_l, (P.k0 + k_l) / P.pps, i_l, sp_l < npk && i_l < W);
+          for (uint32_t x = 0; x < pk_Bp && q0 + x < npk; ++x) {
+            uint64_t r, st, gbad, pbad;
+            batch_masks<AGG | BCAST>(P, d, kfirst + q0 + x, (int)(x * pk_Wp), pk_wmask, r, st, gbad, pbad);
+            if ((uint32_t)lane == x) report(q0 + x, r, st, gbad, pbad);
+          }
+        }
+      } else if (widx < npk * P.P && widx == my_sp * P.P) {
+        uint64_t r, st, gbad, pbad;
+        packet_masks<AGG | BCAST>(P, kfirst + my_sp, (P.k0 + kfirst + my_sp) / P.pps, lane, r, st, gbad, pbad);
+        if (lane == 0) report(my_sp, r, st, gbad, pbad);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(mask_bar(buf));
+    };
+    if constexpr (PACKED) {
+      if (blockIdx.x < G.num_tiles) eval_masks(blockIdx.x, 0u);
+    }
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
-      // PACKED: this warp's 128 elements lie in one small packet; the warp evaluates that packet's masks
-      // itself, before it waits for the tile's data
       uint64_t my_recv = 0, my_stale = 0;
-      uint32_t my_sp = 0;
       bool my_first = false;
       if constexpr (PACKED) {
         const uint32_t kfirst = tile * G.packets_per_tile;
         const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
         const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;
+        // the next tile's masks first (their latency hides behind this tile), then wait for this tile's
+        if (tile + gridDim.x < G.num_tiles) eval_masks(tile + gridDim.x, mbuf ^ 1u);
+        if (!mbar_wait(mask_bar(mbuf), mpar, abort_flag)) { ok = false; break; }
         if (widx < npk * P.P) {
-          my_sp = widx / P.P;
           my_first = widx == my_sp * P.P;
-          const uint32_t k = kfirst + my_sp;
-          uint64_t gbad = 0, pbad = 0;
-          packet_masks<AGG | BCAST>(P, k, (P.k0 + k) / P.pps, lane, my_recv, my_stale, gbad, pbad);
-          if (my_first && lane == 0) {
-            if (P.count) P.count[k] = (uint8_t)__popcll(my_recv);
-            if (P.recv_bits) P.recv_bits[k] = my_recv;
-            if (P.stale_bits) P.stale_bits[k] = my_stale;
-            if (P.burst_out) {
-              P.burst_out[k] = gbad;
-              P.burst_out[(size_t)P.K + k] = pbad;
-            }
-          }
+          my_recv = tmasks[mbuf].recv[my_sp];
+          my_stale = tmasks[mbuf].stale[my_sp];
           if constexpr (DRIFTK) {
             uint64_t sm = my_stale;
             while (sm) {
@@ -555,6 +606,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             }
           }
         }
+        if (++mbuf == 2u) { mbuf = 0; mpar ^= 1u; }
       }
       for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
         if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
