@@ -17,7 +17,7 @@
 // or 8), PRE (how the old copies of stale replicas are read: 0 = by the compute warps in the drift phase, 16 =
 // the first ones requested before the tile's arithmetic into 16 registers per lane, 1 = as extra pipeline
 // stages), PACKED (packets shorter than a tile: several whole packets per tile, masks evaluated by the
-// compute warps) and SPLIT (theta / m / v and the wire tile in two state slots of their own, stages of
+// compute warps a tile ahead) and SPLIT (theta / m / v and the wire tile in two state slots of their own, stages of
 // gradient slots only).
 // Drift norms are finalised by the last CTA to finish (fence + ticket counter; nothing waits on another CTA).
 //
@@ -62,9 +62,10 @@ struct TmaGeom {
 // PACKED build, for packets shorter than a tile: a tile holds up to kMaxSub whole packets. The producer
 // fetches every worker's piece of the tile in ONE bulk copy each (bulk copies under ~2 KB run far below the
 // memory rate, and a single warp cannot evaluate eight packets' masks per tile fast enough); the masks are
-// evaluated by the compute warps instead, each for the one packet its 128 elements lie in, so dropped
-// sub-packets are fetched but never used. The store warp writes each replica the runs of consecutive
-// sub-packets whose broadcast it received.
+// evaluated by the compute warps instead, which split a tile's sub-packets among themselves one tile ahead and
+// share the result in shared memory, so dropped sub-packets are fetched but never used. A compute warp's 128
+// elements lie in one sub-packet, whose masks it reads from there. The store warp writes each replica the
+// runs of consecutive sub-packets whose broadcast it received.
 constexpr int kMaxSub = 8;
 struct __align__(16) PackedStale { uint64_t stale[kMaxSub]; };
 struct __align__(16) PackedMasks { uint64_t recv[kMaxSub], stale[kMaxSub]; };   // a tile's masks, shared by its compute warps
