@@ -422,13 +422,12 @@ int try_phase_tma(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blo
 }
 
 // One single-phase call: complete packets through the bulk-copy pipeline where a build fits (packets of at
-// least one tile, not Algorithm 1's aggregate), a ragged last packet or everything else through the register
-// kernel. With drift norms, pass 0 only sizes the grids: the blocks of both launches draw tickets from one
+// least one tile), a ragged last packet or everything else through the register kernel. With drift norms, pass 0 only sizes the grids: the blocks of both launches draw tickets from one
 // counter and the last of them finalises the norms.
 template <int PH>
 int run_phase(lossy_ctx* ctx, const Params& P, float* norms, double* sumsq, cudaStream_t s) {
   const lossy_config& c = ctx->cfg;
-  const bool bulk = !(c.flags & LOSSY_REGISTER_PATH) && !P.ghat_prev;
+  const bool bulk = !(c.flags & LOSSY_REGISTER_PATH);
   // wide tiles (one CTA per SM) when they divide the packet and the streamed arrays fit two groups
   const bool wide = c.packet_elems % TmaShape<16>::kTile == 0 && c.W <= 16;
   uint32_t tma_blocks = 0, tail_blocks = 0;

@@ -10,7 +10,8 @@
 //   STEP  : ghat, theta (and m, v) in, updated in place, theta (and m, v) out
 //   BCAST : theta in, rounded to the wire type once, one bulk store per replica that receives it
 //   DRIFT : theta and groups of up to GS replica pieces in, squared differences accumulated, nothing out
-// Packets shorter than a tile and a ragged last packet stay on the register kernel.
+// Packets shorter than a tile and a ragged last packet stay on the register kernel. Algorithm 1's aggregate
+// (P.ghat_prev set) runs here too: one draw per packet, the saved aggregate read or written by the compute warps.
 #pragma once
 #include "lossy_tma.cuh"
 
@@ -84,7 +85,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     const uint64_t pol = policy_evict_first();
     constexpr bool kMasked = PH == AGG || PH == BCAST;
     uint32_t Wp = 32;
-    if (kMasked && W <= 16) { Wp = 1; while (Wp < W) Wp <<= 1; }
+    const bool batched = kMasked && W <= 32 && !(PH == AGG && P.ghat_prev);   // Algorithm 1 draws once per packet
+    if (batched && W <= 16) { Wp = 1; while (Wp < W) Wp <<= 1; }
     const uint32_t lgWp = 31u - (uint32_t)__clz((int)Wp);
     const uint32_t B = 32u >> lgWp;                                // tiles per batch
     const uint32_t wmask = Wp == 32 ? 0xFFFFFFFFu : ((1u << Wp) - 1u);
@@ -99,7 +101,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       const uint32_t j_l = (P.k0 + k_l) / P.pps;
       BatchDraws draws = {0u, 0u, 0u};         // W <= 32: one bit per (tile of the batch, worker)
       if constexpr (kMasked) {
-        if (W <= 32) draws = batch_draws<PH>(P, k_l, j_l, i_l, tv && i_l < W);
+        if (batched) draws = batch_draws<PH>(P, k_l, j_l, i_l, tv && i_l < W);
       }
       for (uint32_t b = 0; ok && b < B; ++b) {
         const uint32_t tile = tile0 + b * gridDim.x;
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
         uint32_t cnt = 1;
         if constexpr (kMasked) {
-          if (W <= 32) {
+          if (batched) {
             batch_masks<PH>(P, draws, k, src, wmask, recv, stale, gbad, pbad);
           } else {
             packet_masks<PH>(P, k, j, lane, recv, stale, gbad, pbad);
@@ -256,6 +258,18 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               }
             if (g + 1 == G.groups) {
               divide_by_count<kEpl>(acc, h.cnt);
+              if (P.ghat_prev) {
+                // Algorithm 1: a dropped packet falls back to the saved aggregate, a surviving one is saved
+                uint32_t pw[4];
+                if (h.cnt == 0) {
+                  load_words_stream<kEpl>(P.ghat_prev + h.e0 + idx, pw);
+                  unpack_lane<F32>(pw, acc);
+                } else {
+#pragma unroll
+                  for (int x = 0; x < kEpl; ++x) pw[x] = __float_as_uint(acc[x]);
+                  __stcs(reinterpret_cast<uint4*>(P.ghat_prev + h.e0 + idx), make_uint4(pw[0], pw[1], pw[2], pw[3]));
+                }
+              }
               sts_lane_f32(st + off_tail, idx, acc);
             }
           }
