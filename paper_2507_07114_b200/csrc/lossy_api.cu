@@ -267,13 +267,13 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   }
   if (ctx->cfg.packet_elems < (uint32_t)TmaShape<8>::kTile) {
     // Packets shorter than a tile: the PACKED builds, where they beat the register kernel. They fetch the
-    // dropped sub-packets too, so they win at low loss (+8..17 % at W = 8-16, P = 256-512, p <= 0.1) and lose
-    // at p >= 0.2 from W = 16 and at p >= 0.1 from W = 32; with 2..8 workers they win at every loss rate
+    // dropped sub-packets too, so they win at low loss (+8..17 % at W = 8-16, P = 256-512, p <= 0.1; +3..5 % at
+    // p = 0.2) and lose at p = 0.3 from W = 16 and at p >= 0.1 from W = 32; with 2..8 workers they win at every loss rate
     // (+1..13 %); below 256 elements the register kernel's 256-element chunks are mostly idle lanes and the
     // PACKED build always wins.
     const lossy_config& c = ctx->cfg;
     const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
-    if (c.packet_elems < 256 || (c.W >= 2 && c.W <= 8) || (pm <= 0.15 && c.W <= 24) || (pm <= 0.075 && c.W <= 32)) {
+    if (c.packet_elems < 256 || (c.W >= 2 && c.W <= 8) || (pm <= 0.2 && c.W <= 24) || (pm <= 0.075 && c.W <= 32)) {
       if (c.W <= 16) {
         int rc = try_tma<16, 8, 0, true>(ctx, P, drift, s, blocks, used);
         if (rc || *used) return rc;
