@@ -24,7 +24,8 @@
  *   - Return value: LOSSY_OK or an error code; nothing throws, nothing traps on
  *     the device. A bad argument is rejected before any launch.
  *   - A context owns scratch that its calls share (partial sums, a block counter):
- *     issue the calls of one context on one stream, or order them with events.
+ *     issue the calls of one context on one stream, or order them with events,
+ *     and from one host thread at a time (different contexts are independent).
  *   - The bucket is cut into K = ceil(n / packet_elems) packets of
  *     `packet_elems` contiguous elements (the last may be short). Shard j, owned
  *     by worker j, is the contiguous packet range [j*pps, min(K,(j+1)*pps)) with
