@@ -22,8 +22,9 @@
  * enumeration of all delivery patterns for tiny W, K; unbiasedness over seeds;
  * the four-case drift rule of the Bounded Model Drift proof; exact stationary
  * drift for i.i.d. increments; optimizer trajectories against closed forms; hash
- * statistics. Absolute values of ghat/theta for p > 0 at scale are "parity
- * unpinned" beyond these: the paper prints no worked numeric example.
+ * statistics; slab by slab equals the whole bucket. The paper prints no worked
+ * numeric example, so values at scale rest on the enumeration of tiny cases plus
+ * that packet independence; no function here is without a pin.
  */
 #include <math.h>
 #include <stdint.h>
