@@ -40,7 +40,11 @@ typedef float REAL;
 
 enum { DT_F32 = 0, DT_BF16 = 1 };
 enum { OPT_SGD = 0, OPT_ADAM = 1 };
-enum { FLAG_SELF_LOSSLESS = 1u, FLAG_ZERO_SKIP = 2u };
+enum { FLAG_SELF_LOSSLESS = 1u, FLAG_ZERO_SKIP = 2u,
+       /* Section 3 step (4) sends a shard's update "to all OTHER workers": worker i never needs a replica of
+        * its own shard (what it owns IS the master). With this flag replicas[i] holds only the packets that
+        * worker i does not own, in bucket order, back to back. */
+       FLAG_REPLICA_SKIP_OWNER = 8u };
 
 typedef struct {
   uint32_t W;            /* workers = shards = replicas (paper's N)                    */
@@ -120,7 +124,8 @@ uint32_t NAME(owner)(const oracle_config* c, uint64_t k) {
  *
  *   grads[i]        worker i's gradient slab (cfg.grad_dtype), read only
  *   master, m, v    REAL [n_slab], updated in place (m, v ignored for SGD)
- *   replicas[i]     worker i's copy of the slab (cfg.replica_dtype), updated in place
+ *   replicas[i]     worker i's copy of the slab (cfg.replica_dtype), updated in place; with
+ *                   FLAG_REPLICA_SKIP_OWNER the slab's packets that worker i does not own, back to back
  *   ghat_prev       NULL: Section 3's per-link loss (the default). Non-NULL (REAL [n_slab], in/out):
  *                   Algorithm 1's gradient half — the reduce over all W workers is reliable,
  *                   then ONE draw per packet decides whether the owner keeps the fresh aggregate
@@ -173,6 +178,11 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
   const REAL omb1 = (REAL)1 - b1, omb2 = (REAL)1 - b2;
   const REAL ibc1 = (REAL)(1.0 / (1.0 - pow((double)c->beta1, (double)step)));
   const REAL ibc2 = (REAL)(1.0 / (1.0 - pow((double)c->beta2, (double)step)));
+
+  /* owner-elided replicas: where the current packet starts inside replicas[i] */
+  const int elide = (c->flags & FLAG_REPLICA_SKIP_OWNER) != 0;
+  uint64_t cursor[64];
+  for (uint32_t i = 0; i < 64; ++i) cursor[i] = 0;
 
   for (uint64_t kl = 0; kl < packets; ++kl) {
     const uint64_t k = k0 + kl;                 /* packet within the bucket */
@@ -284,17 +294,21 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
       const uint16_t wire_h = NAME(f32_to_bf16)(wire_f);
       const double x = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(wire_h) : (double)wire_f;
       for (uint32_t i = 0; i < W; ++i) {
+        if (elide && i == j) continue;           /* the owner keeps no replica of its own shard: drift term 0 */
+        const uint64_t at = elide ? cursor[i] + (e - e0) : e;
         if (!((stale >> i) & 1ULL)) {
-          if (c->replica_dtype == DT_BF16) ((uint16_t*)replicas[i])[e] = wire_h;
-          else ((float*)replicas[i])[e] = wire_f;
+          if (c->replica_dtype == DT_BF16) ((uint16_t*)replicas[i])[at] = wire_h;
+          else ((float*)replicas[i])[at] = wire_f;
         } else if (sumsq) {
-          double r = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[e])
-                                                 : (double)((const float*)replicas[i])[e];
+          double r = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[at])
+                                                 : (double)((const float*)replicas[i])[at];
           double d = r - x;
           sumsq[i] += d * d;
         }
       }
     }
+    for (uint32_t i = 0; i < W; ++i)
+      if (i != j) cursor[i] += e1 - e0;
     if (age)
       for (uint32_t i = 0; i < W; ++i) age[i][kl] = ((stale >> i) & 1ULL) ? age[i][kl] + 1u : 0u;
   }
@@ -304,16 +318,24 @@ int NAME(step)(const oracle_config* c, uint64_t step, uint64_t k0, uint64_t n_sl
 /*
  * Drift of every replica from the owners' current values, on its own (no
  * broadcast): sumsq[i] += sum_e (replica_i[e] - cast(master[e]))^2 in double.
+ * The slab starts at bucket packet k0 (only the owner-elided layout needs it: there
+ * worker i has no copy of its own packets, which add nothing to its sum).
  */
-int NAME(drift_sumsq)(const oracle_config* c, uint64_t n_slab, const REAL* master,
+int NAME(drift_sumsq)(const oracle_config* c, uint64_t k0, uint64_t n_slab, const REAL* master,
                       const void* const* replicas, double* sumsq) {
   if (!c || !sumsq) return 1;
+  const int elide = (c->flags & FLAG_REPLICA_SKIP_OWNER) != 0;
+  uint64_t at[64];                               /* next element of replicas[i] */
+  for (uint32_t i = 0; i < 64; ++i) at[i] = 0;
   for (uint64_t e = 0; e < n_slab; ++e) {
+    const uint32_t j = NAME(owner)(c, k0 + e / c->packet_elems);
     const float wire_f = (float)master[e];
     const double x = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(NAME(f32_to_bf16)(wire_f)) : (double)wire_f;
     for (uint32_t i = 0; i < c->W; ++i) {
-      double r = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[e])
-                                             : (double)((const float*)replicas[i])[e];
+      if (elide && i == j) continue;
+      const uint64_t q = at[i]++;
+      double r = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[q])
+                                             : (double)((const float*)replicas[i])[q];
       double d = r - x;
       sumsq[i] += d * d;
     }
@@ -331,6 +353,7 @@ int NAME(drift_sumsq)(const oracle_config* c, uint64_t n_slab, const REAL* maste
 int NAME(closed_loop_grads)(const oracle_config* c, uint64_t n_slab, const float* curv, const float* target,
                             const void* const* noise, const void* const* replicas, void* const* grads_out) {
   if (!c || !curv || !target || !noise || !replicas || !grads_out) return 1;
+  if (c->flags & FLAG_REPLICA_SKIP_OWNER) return 1;   /* needs every worker's full copy */
   for (uint32_t i = 0; i < c->W; ++i)
     for (uint64_t e = 0; e < n_slab; ++e) {
       REAL rep = c->replica_dtype == DT_BF16 ? (REAL)bf16_to_f32(((const uint16_t*)replicas[i])[e])
@@ -348,20 +371,31 @@ int NAME(closed_loop_grads)(const oracle_config* c, uint64_t n_slab, const float
  * The theorem's own quantity ("Quantifying Model Drift": D = theta^(i,j) - theta^(k,j) between two
  * workers' copies): d2[i*W + k] += sum_e (replica_i[e] - replica_k[e])^2 for every pair, in double.
  */
-int NAME(pairwise_sumsq)(const oracle_config* c, uint64_t n_slab, const void* const* replicas, double* d2) {
+int NAME(pairwise_sumsq)(const oracle_config* c, uint64_t k0, uint64_t n_slab, const void* const* replicas, double* d2) {
   if (!c || !replicas || !d2) return 1;
   const uint32_t W = c->W;
-  for (uint64_t e = 0; e < n_slab; ++e)
+  /* Owner-elided layout: the owner of an element holds no replica of it, so on that element the sums run
+   * over the pairs of the other workers only (the theorem's D is between two receivers of shard j). */
+  const int elide = (c->flags & FLAG_REPLICA_SKIP_OWNER) != 0;
+  uint64_t at[64];
+  for (uint32_t i = 0; i < 64; ++i) at[i] = 0;
+  for (uint64_t e = 0; e < n_slab; ++e) {
+    const uint32_t j = NAME(owner)(c, k0 + e / c->packet_elems);
     for (uint32_t i = 0; i < W; ++i) {
-      double ri = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[e])
-                                              : (double)((const float*)replicas[i])[e];
+      if (elide && i == j) continue;
+      double ri = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[i])[at[i]])
+                                              : (double)((const float*)replicas[i])[at[i]];
       for (uint32_t k = 0; k < W; ++k) {
-        double rk = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[k])[e])
-                                                : (double)((const float*)replicas[k])[e];
+        if (elide && k == j) continue;
+        double rk = c->replica_dtype == DT_BF16 ? (double)bf16_to_f32(((const uint16_t*)replicas[k])[at[k]])
+                                                : (double)((const float*)replicas[k])[at[k]];
         double d = ri - rk;
         d2[(size_t)i * W + k] += d * d;
       }
     }
+    for (uint32_t i = 0; i < W; ++i)
+      if (!(elide && i == j)) at[i]++;
+  }
   return 0;
 }
 

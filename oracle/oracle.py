@@ -27,7 +27,7 @@ _libs: dict = {}
 
 F32, BF16 = 0, 1
 SGD, ADAM = 0, 1
-SELF_LOSSLESS, ZERO_SKIP = 1, 2
+SELF_LOSSLESS, ZERO_SKIP, REPLICA_SKIP_OWNER = 1, 2, 8
 
 
 class OracleConfig(C.Structure):
@@ -81,7 +81,7 @@ def _lib(f64: bool):
         s.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64] + [C.c_void_p] * 18
         ds = getattr(lib, pre + "drift_sumsq")
         ds.restype = C.c_int
-        ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
+        ds.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
         mk = getattr(lib, pre + "masks")
         mk.restype = C.c_int
         mk.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -90,7 +90,7 @@ def _lib(f64: bool):
         sq.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p]
         pw = getattr(lib, pre + "pairwise_sumsq")
         pw.restype = C.c_int
-        pw.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_void_p, C.c_void_p]
+        pw.argtypes = [C.POINTER(OracleConfig), C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
         cl = getattr(lib, pre + "closed_loop_grads")
         cl.restype = C.c_int
         cl.argtypes = [C.POINTER(OracleConfig), C.c_uint64] + [C.c_void_p] * 5
@@ -158,7 +158,9 @@ class Oracle:
         self.m = np.zeros(self.n_slab, self.real)
         self.v = np.zeros(self.n_slab, self.real)
         wire = cast_wire(theta0, replica_dtype)
-        self.replicas = [wire.copy() for _ in range(W)]
+        self.elided = bool(flags & REPLICA_SKIP_OWNER)
+        # owner-elided layout: worker i's array holds the slab without the packets it owns, back to back
+        self.replicas = [wire[self.kept(i)].copy() if self.elided else wire.copy() for i in range(W)]
         self.age = [np.zeros(self.packets, np.uint32) for _ in range(W)] if track_age else None
         # Algorithm 1's gradient half keeps the last surviving aggregate per element ("g_prev"), zero at start
         self.ghat_prev = np.zeros(self.n_slab, self.real) if alg1 else None
@@ -169,6 +171,14 @@ class Oracle:
 
     def owner(self, k: int) -> int:
         return getattr(self.lib, self.pre + "owner")(C.byref(self.cfg), k)
+
+    def kept(self, i: int) -> np.ndarray:
+        """Boolean mask over the slab's elements: True where worker i is NOT the owner (what its array
+        holds in the owner-elided layout)."""
+        K = (self.n + self.P - 1) // self.P
+        pps = (K + self.W - 1) // self.W
+        owner_of_elem = (self.k0 + np.arange(self.n_slab, dtype=np.int64) // self.P) // pps
+        return owner_of_elem != i
 
     def set_lr(self, lr: float) -> None:
         self.cfg.lr = lr
@@ -250,8 +260,8 @@ class Oracle:
         """W x W matrix of sum_e (replica_i[e] - replica_k[e])^2, in double (the theorem's pairwise drift)."""
         d2 = np.zeros((self.W, self.W), np.float64)
         rt = _ptr_table(self.replicas)
-        rc = getattr(self.lib, self.pre + "pairwise_sumsq")(C.byref(self.cfg), self.n_slab, C.cast(rt, C.c_void_p),
-                                                            _ptr(d2))
+        rc = getattr(self.lib, self.pre + "pairwise_sumsq")(C.byref(self.cfg), self.k0, self.n_slab,
+                                                            C.cast(rt, C.c_void_p), _ptr(d2))
         if rc != 0:
             raise ValueError("oracle_pairwise_sumsq rejected its arguments")
         return d2
@@ -261,7 +271,7 @@ class Oracle:
         sumsq = np.zeros(self.W, np.float64)
         rt = _ptr_table(self.replicas)
         rc = getattr(self.lib, self.pre + "drift_sumsq")(
-            C.byref(self.cfg), self.n_slab, _ptr(self.master), C.cast(rt, C.c_void_p), _ptr(sumsq))
+            C.byref(self.cfg), self.k0, self.n_slab, _ptr(self.master), C.cast(rt, C.c_void_p), _ptr(sumsq))
         if rc != 0:
             raise ValueError("oracle_drift_sumsq rejected its arguments")
         return sumsq

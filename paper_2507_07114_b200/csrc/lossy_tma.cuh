@@ -541,7 +541,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     const uint32_t pk_Bp = min(32u >> pk_lgWp, 2u);
     const uint32_t pk_wmask = pk_Wp == 32 ? 0xFFFFFFFFu : ((1u << pk_Wp) - 1u);
     // PACKED: a tile's masks are evaluated once, one tile ahead, and shared through two alternating buffers
-    // (a warp that is ahead never overwrites masks still being read): with W <= 32 (not Algorithm 1) warp w
+    // (the main loop reads a tile's masks before it writes the next tile's, which is what keeps a warp that
+    // is ahead from overwriting masks still to be read): with W <= 32 (not Algorithm 1) warp w
     // takes the w-th batch of 32 / Wp sub-packets in one pass of draws; otherwise the first warp of each
     // sub-packet takes its own. Every compute warp arrives on the buffer's barrier once per tile.
     auto eval_masks = [&](uint32_t tile, uint32_t buf) {
@@ -591,13 +592,20 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint32_t kfirst = tile * G.packets_per_tile;
         const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
         const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;
-        // the next tile's masks first (their latency hides behind this tile), then wait for this tile's
-        if (tile + gridDim.x < G.num_tiles) eval_masks(tile + gridDim.x, mbuf ^ 1u);
+        // This tile's masks (written one iteration ago) are copied to registers BEFORE the next tile's are
+        // written into the other buffer. Order of events per warp and iteration n: wait(n), read(n), write(n+1),
+        // arrive(n+1). A warp's wait(n) therefore proves that every warp has arrived for tile n, i.e. has
+        // finished read(n-1) — so write(n+1), which reuses the buffer of tile n-1, overwrites nothing that is
+        // still to be read, however far the warps of a CTA drift apart inside a tile.
         if (!mbar_wait(mask_bar(mbuf), mpar, abort_flag)) { ok = false; break; }
         if (widx < npk * P.P) {
           my_first = widx == my_sp * P.P;
           my_recv = tmasks[mbuf].recv[my_sp];
           my_stale = tmasks[mbuf].stale[my_sp];
+        }
+        // the next tile's masks now: their latency hides behind this tile's pipeline waits
+        if (tile + gridDim.x < G.num_tiles) eval_masks(tile + gridDim.x, mbuf ^ 1u);
+        if (widx < npk * P.P) {
           if constexpr (DRIFTK) {
             uint64_t sm = my_stale;
             while (sm) {
