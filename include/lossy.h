@@ -25,7 +25,12 @@
  *     the device. A bad argument is rejected before any launch.
  *   - A context owns scratch that its calls share (partial sums, a block counter):
  *     issue the calls of one context on one stream, or order them with events,
- *     and from one host thread at a time (different contexts are independent).
+ *     and from one host thread at a time. Different contexts are independent and
+ *     may be driven from different host threads (the little process-wide state the
+ *     launches share is locked inside the library).
+ *   - After LOSSY_ECUDA the context stays usable only if the CUDA error was not
+ *     sticky (a failed launch configuration is not; a device fault is): check the
+ *     runtime's own error state before going on.
  *   - The bucket is cut into K = ceil(n / packet_elems) packets of
  *     `packet_elems` contiguous elements (the last may be short). Shard j, owned
  *     by worker j, is the contiguous packet range [j*pps, min(K,(j+1)*pps)) with
@@ -66,7 +71,19 @@ enum {
    * the tile and the measured policy favours it (few workers, or low loss; that build also
    * fetches the dropped packets of a tile). Same parameters, replicas and masks either way; drift
    * sums agree to rounding (another summation order). */
-  LOSSY_REGISTER_PATH = 4u
+  LOSSY_REGISTER_PATH = 4u,
+  /* Owner-elided replicas. Section 3 step (4) sends a shard's new values "to all OTHER workers": the
+   * owner of a shard needs no replica of it (what it owns is the master copy, and its drift term is
+   * exactly 0). With this flag replica i holds the bucket WITHOUT the packets worker i owns: the
+   * elements in front of worker i's shard keep their index, the elements behind it sit
+   * |shard i| elements lower, and the array has lossy_replica_elems(ctx, i) elements (n minus the
+   * shard). Every entry point that takes `replicas` reads and writes this layout; masks, counts,
+   * parameters, moments, every element a worker does not own and the drift norms are the same as
+   * without the flag. It saves 1/W of the replica memory (a full 7B-parameter model with W = 8 then
+   * fits one 180 GB GPU). A replica that would hold nothing (W = 1) may be NULL.
+   * drift_pairwise then sums, on every element, over the pairs of workers that both hold a copy;
+   * lossy_closed_loop_grads needs full replicas and rejects such a context. */
+  LOSSY_REPLICA_SKIP_OWNER = 8u
 };
 
 #define LOSSY_MAX_WORKERS 64u
@@ -82,7 +99,7 @@ typedef struct {
   uint32_t grad_dtype;   /* LOSSY_F32 or LOSSY_BF16                                     */
   uint32_t replica_dtype;/* LOSSY_F32 or LOSSY_BF16 (bf16 = round-to-nearest-even cast) */
   uint32_t optimizer;    /* LOSSY_SGD or LOSSY_ADAM                                     */
-  uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH */
+  uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH, LOSSY_REPLICA_SKIP_OWNER */
   float lr, beta1, beta2, eps; /* eta_t and Adam's constants (beta/eps unused for SGD)  */
   /* Packet-range sharding (several GPUs simulate one bucket, each a contiguous range of its
    * packets for all W workers): this context's packet 0 is packet shard_packet0 of a bucket of
@@ -184,7 +201,10 @@ int lossy_aggregate(lossy_ctx* ctx, uint64_t step, const void* const* grads,
  *         theta = theta - (lr * (m*ibc1)) / (sqrt(v*ibc2) + eps)
  *         ibc1 = float(1/(1-b1^step)), ibc2 = float(1/(1-b2^step)) from double on the host.
  *   count      [K] uint8 from lossy_aggregate; needed (non-NULL) only with
- *              LOSSY_ZERO_SKIP, where packets with count 0 are left untouched
+ *              LOSSY_ZERO_SKIP, where packets with count 0 are left untouched. (The update
+ *              as the paper prints it needs only ghat; this one argument carries the
+ *              "nothing arrived" fact from the aggregate to the update when the two are
+ *              separate calls, which the fused call knows by itself.)
  *   master     [n] fp32, updated in place;  m, v: [n] fp32 (Adam only, else NULL)
  */
 int lossy_step(lossy_ctx* ctx, uint64_t step, const float* ghat, const uint8_t* count,
@@ -196,8 +216,10 @@ int lossy_step(lossy_ctx* ctx, uint64_t step, const float* ghat, const uint8_t* 
  *     hash(seed, step, src=owner, dst=i, packet_base+k) >= T_param,
  * otherwise the replica's packet is left exactly as it was (stale).
  *   master     [n] fp32 (read only)
- *   replicas   host array of W device pointers, each [n] of cfg.replica_dtype
+ *   replicas   host array of W device pointers, each [n] of cfg.replica_dtype (with
+ *              LOSSY_REPLICA_SKIP_OWNER: [lossy_replica_elems(ctx, i)], see the flag)
  *   stale_bits [K] uint64, written (bit i = replica i kept its old packet), or NULL
+ * `step` must be >= 1 here and in lossy_aggregate too (LOSSY_EINVAL otherwise).
  */
 int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master,
                     void* const* replicas, uint64_t* stale_bits, void* stream);
@@ -242,7 +264,9 @@ int drift_pairwise(lossy_ctx* ctx, const void* const* replicas, double* d2, void
  * cudaFree or other allocating routine.
  *
  *   cfg       host pointer; W, n, packet_elems and replica_dtype are used (the
- *             chunks of the reduction follow the packet grid), the rest is ignored
+ *             chunks of the reduction follow the packet grid), and of the flags
+ *             LOSSY_REPLICA_SKIP_OWNER with shard_packet0 / bucket_packets (the
+ *             replica layout depends on the shard map); the rest is ignored
  *   master    [n] fp32 device;  replicas: host array of W device pointers, each [n]
  *   norms     [W] fp32 device, written, or NULL;  sumsq: [W] fp64 device, ADDED to,
  *             or NULL (at least one of the two)
@@ -252,7 +276,11 @@ int drift_pairwise(lossy_ctx* ctx, const void* const* replicas, double* d2, void
  * nothing. The grid is capped at the 1024 rows of the static array.
  * First call on a device: looks up the device address of the static array
  * (cudaGetSymbolAddress, with that device current) and caches it; make that
- * first call before any stream capture begins.
+ * first call at start-up, before any stream capture begins and before the
+ * process commits or freezes the rest of its device memory: CUDA loads a
+ * library's device code on first use, and that first use is what reserves the
+ * kernels' and the array's memory (LOSSY_ENOMEM if there is no room for it).
+ * The cached address does not survive a cudaDeviceReset of that device.
  * Sharing: every call in the process uses the same array and finds the last
  * call's contents in it; each call overwrites every row it later reads, so
  * nothing needs clearing, but two calls that overlap on the GPU (different
@@ -347,8 +375,32 @@ int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* targ
  * on its barriers instead of spinning forever). LOSSY_OK, or LOSSY_EDEVICE if
  * the results of an earlier call on this context must be discarded. The paper
  * has no counterpart; this is the library's failure report.
+ * The status word is sticky: once set it stays set, and every later
+ * lossy_device_status on the context returns LOSSY_EDEVICE, until
+ * lossy_reset_status clears it.
  */
 int lossy_device_status(lossy_ctx* ctx, void* stream);
+
+/*
+ * lossy_reset_status — clear the context's device status word and its
+ * finished-block counter on `stream` (asynchronous), so that the context can be
+ * used again after a reported LOSSY_EDEVICE. The state arrays of the step that
+ * reported it (master, m, v, replicas) are the caller's to restore, e.g. from a
+ * checkpoint: a kernel that gave up may have updated some tiles and not others.
+ * The paper has no counterpart.
+ */
+int lossy_reset_status(lossy_ctx* ctx, void* stream);
+
+/*
+ * lossy_selftest_wait_expiry — exercise the failure report without a failure.
+ * Launches one small thread block that waits, with the pipelines' own bounded
+ * wait and a poll limit of `max_polls` (1 .. 2^20), on a barrier that nothing
+ * will ever complete; no copy is in flight. The wait runs out, the block leaves
+ * through the pipelines' exit path and sets this context's status word, so the
+ * next lossy_device_status returns LOSSY_EDEVICE. Nothing faults, traps or hangs,
+ * and the device context stays usable. A test hook; the paper has no counterpart.
+ */
+int lossy_selftest_wait_expiry(lossy_ctx* ctx, uint32_t max_polls, void* stream);
 
 /*
  * lossy_mask — host evaluation of one delivery indicator of Section 3:
@@ -381,6 +433,10 @@ const char* lossy_last_error(const lossy_ctx* ctx);
 
 /* lossy_num_packets — K = ceil(n / packet_elems) for this context (0 for NULL). */
 uint64_t lossy_num_packets(const lossy_ctx* ctx);
+
+/* lossy_replica_elems — elements replica `worker`'s array holds: n, or with LOSSY_REPLICA_SKIP_OWNER n minus
+ * the elements of that worker's own shard inside this context's packet range (0 for NULL or worker >= W). */
+uint64_t lossy_replica_elems(const lossy_ctx* ctx, uint32_t worker);
 
 /* lossy_kernel_launches — kernels this context has launched so far (0 for NULL). */
 uint64_t lossy_kernel_launches(const lossy_ctx* ctx);

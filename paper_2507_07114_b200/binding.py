@@ -17,13 +17,13 @@ from . import build as _build
 LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE, LOSSY_ELIMIT = 0, 1, 2, 3, 4, 5
 LOSSY_F32, LOSSY_BF16 = 0, 1
 LOSSY_SGD, LOSSY_ADAM = 0, 1
-LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH = 1, 2, 4
+LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH, LOSSY_REPLICA_SKIP_OWNER = 1, 2, 4, 8
 
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_set_reliable", "lossy_packet_sqnorms", "lossy_aggregate", "lossy_step", "lossy_broadcast",
     "drift_norms", "drift_pairwise", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
-    "lossy_describe_plan",
+    "lossy_describe_plan", "lossy_replica_elems", "lossy_reset_status", "lossy_selftest_wait_expiry",
 ]
 
 
@@ -105,6 +105,12 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_num_packets.argtypes = [vp]
     lib.lossy_kernel_launches.restype = u64
     lib.lossy_kernel_launches.argtypes = [vp]
+    lib.lossy_replica_elems.restype = u64
+    lib.lossy_replica_elems.argtypes = [vp, u32]
+    lib.lossy_reset_status.restype = C.c_int
+    lib.lossy_reset_status.argtypes = [vp, vp]
+    lib.lossy_selftest_wait_expiry.restype = C.c_int
+    lib.lossy_selftest_wait_expiry.argtypes = [vp, u32, vp]
     lib.lossy_describe_plan.restype = C.c_int
     lib.lossy_describe_plan.argtypes = [vp, C.c_int, C.c_char_p, C.c_size_t]
     if path == _build.LIB_PATH:
@@ -125,7 +131,7 @@ def _p(t):
 
 
 def _table(ts):
-    return (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+    return (C.c_void_p * len(ts))(*[None if t is None else t.data_ptr() for t in ts])
 
 
 def _stream():
@@ -197,17 +203,19 @@ def drift_pairwise(ctx, replicas, d2):
     _check(ctx, load_library().drift_pairwise(ctx, _table(replicas), _p(d2), _stream()))
 
 
-def drift_norms_static(*, W, n, packet_elems, replica_dtype, master, replicas, norms=None, sumsq=None):
+def drift_norms_static(*, W, n, packet_elems, replica_dtype, master, replicas, norms=None, sumsq=None, flags=0,
+                       shard_packet0=0, bucket_packets=0):
     """drift_norms for callers that may not allocate device memory (no context; static scratch in the library).
 
     Raises LossyError with code LOSSY_ELIMIT when a size is beyond the static scratch's limits."""
-    cfg = lossy_config(W, packet_elems, n, 0, 0.0, 0.0, 0, LOSSY_F32, _dt(replica_dtype), LOSSY_SGD, 0,
-                       0.0, 0.0, 0.0, 0.0, 0, 0)
+    cfg = lossy_config(W, packet_elems, n, 0, 0.0, 0.0, 0, LOSSY_F32, _dt(replica_dtype), LOSSY_SGD, flags,
+                       0.0, 0.0, 0.0, 0.0, shard_packet0, bucket_packets)
     rc = load_library().drift_norms_static(C.byref(cfg), _p(master), _table(replicas), _p(norms), _p(sumsq),
                                            _stream())
     if rc != LOSSY_OK:
         raise LossyError(rc, "drift_norms_static: " + {LOSSY_EINVAL: "bad argument", LOSSY_ELIMIT:
-                         "size beyond the static scratch limits", LOSSY_ECUDA: "CUDA error"}.get(rc, "error"))
+                         "size beyond the static scratch limits", LOSSY_ECUDA: "CUDA error",
+                         LOSSY_ENOMEM: "no device memory left to load the library image"}.get(rc, "error"))
 
 
 def lossy_fused_step(ctx, step, grads, master, m, v, replicas, ghat=None, count=None, recv_bits=None,
@@ -259,6 +267,18 @@ def lossy_closed_loop_grads(ctx, curv, target, noise, replicas, grads_out):
 def lossy_device_status(ctx):
     """Synchronise the current stream; raises LossyError(LOSSY_EDEVICE) if a kernel gave up a bounded wait."""
     _check(ctx, load_library().lossy_device_status(ctx, _stream()))
+
+
+def lossy_reset_status(ctx):
+    _check(ctx, load_library().lossy_reset_status(ctx, _stream()))
+
+
+def lossy_selftest_wait_expiry(ctx, max_polls: int = 1024):
+    _check(ctx, load_library().lossy_selftest_wait_expiry(ctx, max_polls, _stream()))
+
+
+def lossy_replica_elems(ctx, worker: int) -> int:
+    return load_library().lossy_replica_elems(ctx, worker)
 
 
 def lossy_last_error(ctx) -> str:

@@ -6,6 +6,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "lossy_phase_tma.cuh"
@@ -59,6 +60,29 @@ int check_table(lossy_ctx* ctx, const void* const* tab, const char* name) {
   return LOSSY_OK;
 }
 
+// elements of worker i's shard inside this context's packet range (what an owner-elided replica leaves out)
+uint64_t own_elems(const lossy_ctx* ctx, uint32_t i) {
+  const lossy_config& c = ctx->cfg;
+  const uint64_t s0 = (uint64_t)i * ctx->pps, s1 = s0 + ctx->pps;
+  const uint64_t c0 = c.shard_packet0, c1 = c.shard_packet0 + ctx->K;
+  const uint64_t lo = s0 > c0 ? s0 : c0, hi = s1 < c1 ? s1 : c1;
+  if (lo >= hi) return 0;
+  const uint64_t e0 = (lo - c0) * c.packet_elems, e1 = (hi - c0) * c.packet_elems;
+  return (e1 < c.n ? e1 : c.n) - (e0 < c.n ? e0 : c.n);
+}
+
+// The replica table: W aligned device pointers; an owner-elided replica that holds nothing may be NULL.
+int check_replicas(lossy_ctx* ctx, const void* const* tab) {
+  const char* name = "replicas: NULL or misaligned pointer";
+  if (!tab) return fail(ctx, LOSSY_EINVAL, name);
+  const bool elide = ctx->cfg.flags & LOSSY_REPLICA_SKIP_OWNER;
+  for (uint32_t i = 0; i < ctx->cfg.W; ++i) {
+    if (elide && own_elems(ctx, i) == ctx->cfg.n) continue;
+    if (!tab[i] || !aligned16(tab[i])) return fail(ctx, LOSSY_EINVAL, name);
+  }
+  return LOSSY_OK;
+}
+
 void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   memset(&P, 0, sizeof P);
   const lossy_config& c = ctx->cfg;
@@ -85,6 +109,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   P.partials = ctx->partials;
   P.K = (uint32_t)ctx->K;
   P.reliable = ctx->reliable;
+  fill_rep_skip(P, (c.flags & LOSSY_REPLICA_SKIP_OWNER) != 0);
   if (ctx->burst_state) {
     // the states after step t-1 live in buffer (t-1)&1, those after step t go to buffer t&1
     const size_t buf = 2 * (size_t)ctx->K;
@@ -139,6 +164,10 @@ TmaPolicy tma_policy(const lossy_config& c) {
 }
 
 constexpr int kMaxDevices = 64;
+// The launch helpers below remember, per kernel instantiation and device, what they set up once (the raised
+// shared-memory limit, the occupancy). Those tables are process-wide, so host threads that drive different
+// contexts take this lock around the look-up; it is never held across a launch.
+std::mutex g_setup_mu;
 
 // Dynamic shared memory one CTA of the bulk-copy kernel may use: the CTAs of one SM share 227 KB.
 template <int CW>
@@ -205,10 +234,13 @@ int launch_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s
   if (ctx->plan_only) return LOSSY_OK;
   static bool opted_in[kMaxDevices];   // per kernel instantiation and device: raise the dynamic shared memory limit once
   cudaError_t e;
-  if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
-    if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
-    if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
+      if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
+      if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+    }
   }
   kern<<<blocks, kThreadsTma, smem, s>>>(P, G);
   e = cudaGetLastError();
@@ -303,14 +335,18 @@ template <int PH, class GT, class RT, int OPT>
 int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out) {
   auto kern = lossy_kernel<PH, GT, RT, OPT>;
   static int occupancy[kMaxDevices];   // per kernel instantiation and device: resident blocks per SM
-  int per_sm = ctx->device < kMaxDevices ? occupancy[ctx->device] : 0;
+  int per_sm = 0;
   cudaError_t e;
-  if (per_sm == 0) {
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, 0);
-    if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
-    if (per_sm < 1) per_sm = 1;
-    if (per_sm > kBlocksPerSmCap) per_sm = kBlocksPerSmCap;
-    if (ctx->device < kMaxDevices) occupancy[ctx->device] = per_sm;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    per_sm = ctx->device < kMaxDevices ? occupancy[ctx->device] : 0;
+    if (per_sm == 0) {
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, 0);
+      if (e != cudaSuccess) return fail_cuda(ctx, "occupancy query", e);
+      if (per_sm < 1) per_sm = 1;
+      if (per_sm > kBlocksPerSmCap) per_sm = kBlocksPerSmCap;
+      if (ctx->device < kMaxDevices) occupancy[ctx->device] = per_sm;
+    }
   }
   uint32_t blocks = (uint32_t)(ctx->num_sms * per_sm);
   const uint32_t need = (P.num_chunks - P.chunk_begin + kWarps - 1) / kWarps;
@@ -391,10 +427,13 @@ int launch_phase_tma(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStre
   if (ctx->plan_only) return LOSSY_OK;
   static bool opted_in[kMaxDevices];   // per kernel instantiation and device: raise the dynamic shared memory limit once
   cudaError_t e;
-  if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
-    if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
-    if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
+      if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
+      if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+    }
   }
   kern<<<blocks, TmaShape<CW>::kThreads, smem, s>>>(P, G);
   e = cudaGetLastError();
@@ -457,7 +496,11 @@ int run_phase(lossy_ctx* ctx, const Params& P, float* norms, double* sumsq, cuda
       else tail_blocks = 0;
     }
     ctx->plan_only = false;
-    if (rc) return rc;
+    if (rc) {
+      // a ticketed launch may already be queued: the counter must be zero again before the next call
+      if (Q.ticket) cudaMemsetAsync(ctx->ticket, 0, sizeof(uint32_t), s);
+      return rc;
+    }
   }
   return LOSSY_OK;
 }
@@ -473,7 +516,8 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   if (cfg->packet_elems == 0 || cfg->packet_elems % 8 != 0) return LOSSY_EINVAL;
   if (!(cfg->p_grad >= 0.0 && cfg->p_grad < 1.0) || !(cfg->p_param >= 0.0 && cfg->p_param < 1.0)) return LOSSY_EINVAL;
   if (cfg->grad_dtype > LOSSY_BF16 || cfg->replica_dtype > LOSSY_BF16 || cfg->optimizer > LOSSY_ADAM) return LOSSY_EINVAL;
-  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH)) return LOSSY_EINVAL;
+  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH | LOSSY_REPLICA_SKIP_OWNER))
+    return LOSSY_EINVAL;
   const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
   const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;
   if (K * cpp >= (1ull << 31)) return LOSSY_EINVAL;  // stream larger models bucket by bucket
@@ -579,6 +623,7 @@ int lossy_set_lr(lossy_ctx* ctx, float lr) {
 static int aggregate_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, float* ghat_prev, float* ghat,
                           uint8_t* count, uint64_t* recv_bits, void* stream) {
   if (ctx->cfg.n == 0) return LOSSY_OK;
+  if (step == 0) return fail(ctx, LOSSY_EINVAL, "step is 1-based");
   if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
   if (!ghat || !aligned16(ghat)) return fail(ctx, LOSSY_EINVAL, "ghat: NULL or misaligned");
   Params P;
@@ -634,7 +679,8 @@ int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master, void* co
                     void* stream) {
   if (!ctx) return LOSSY_EINVAL;
   if (ctx->cfg.n == 0) return LOSSY_OK;
-  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (step == 0) return fail(ctx, LOSSY_EINVAL, "step is 1-based");
+  if (int rc = check_replicas(ctx, replicas)) return rc;
   if (!master || !aligned16(master)) return fail(ctx, LOSSY_EINVAL, "master: NULL or misaligned");
   Params P;
   fill_common(ctx, step, P);
@@ -647,7 +693,7 @@ int lossy_broadcast(lossy_ctx* ctx, uint64_t step, const float* master, void* co
 int drift_norms(lossy_ctx* ctx, const float* master, const void* const* replicas, float* norms, double* sumsq,
                 void* stream) {
   if (!ctx) return LOSSY_EINVAL;
-  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (int rc = check_replicas(ctx, replicas)) return rc;
   if (ctx->cfg.n == 0) {
     if (norms) {
       cudaError_t e = cudaMemsetAsync(norms, 0, ctx->cfg.W * sizeof(float), (cudaStream_t)stream);
@@ -668,7 +714,7 @@ static int fused_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, f
                       uint64_t* stale_bits, float* norms, double* sumsq, void* stream) {
   if (step == 0) return fail(ctx, LOSSY_EINVAL, "step is 1-based");
   if (int rc = check_table(ctx, grads, "grads: NULL or misaligned pointer")) return rc;
-  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (int rc = check_replicas(ctx, replicas)) return rc;
   if (ctx->cfg.n == 0) {
     if (norms) {
       cudaError_t e = cudaMemsetAsync(norms, 0, ctx->cfg.W * sizeof(float), (cudaStream_t)stream);
@@ -727,7 +773,11 @@ static int fused_impl(lossy_ctx* ctx, uint64_t step, const void* const* grads, f
         tail_blocks = 0;
     }
     ctx->plan_only = false;
-    if (rc) return rc;
+    if (rc) {
+      // a ticketed launch may already be queued: the counter must be zero again before the next call
+      if (Q.ticket) cudaMemsetAsync(ctx->ticket, 0, sizeof(uint32_t), s);
+      return rc;
+    }
   }
   return LOSSY_OK;
 }
@@ -752,7 +802,7 @@ int lossy_fused_step_alg1(lossy_ctx* ctx, uint64_t step, const void* const* grad
 int drift_pairwise(lossy_ctx* ctx, const void* const* replicas, double* d2, void* stream) {
   if (!ctx) return LOSSY_EINVAL;
   if (!d2) return fail(ctx, LOSSY_EINVAL, "d2: NULL");
-  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (int rc = check_replicas(ctx, replicas)) return rc;
   if (ctx->cfg.n == 0) return LOSSY_OK;
   PairwiseArgs A;
   memset(&A, 0, sizeof A);
@@ -761,6 +811,13 @@ int drift_pairwise(lossy_ctx* ctx, const void* const* replicas, double* d2, void
   A.n = ctx->cfg.n;
   A.W = ctx->cfg.W;
   A.nblk = (ctx->cfg.W + 3) / 4;
+  if (ctx->cfg.flags & LOSSY_REPLICA_SKIP_OWNER) {
+    A.elide = 1u;
+    A.P = ctx->cfg.packet_elems;
+    A.pps = ctx->pps;
+    A.k0 = (uint32_t)ctx->cfg.shard_packet0;
+    for (uint32_t i = 0; i < ctx->cfg.W; ++i) A.rep_skip[i] = own_elems(ctx, i);
+  }
   const uint32_t pairs = A.nblk * (A.nblk + 1) / 2;
   const uint64_t nvec = (A.n + 7) / 8;
   uint64_t bx = (nvec + 255) / 256;
@@ -780,9 +837,11 @@ int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* targ
                             const void* const* replicas, void* const* grads_out, void* stream) {
   if (!ctx) return LOSSY_EINVAL;
   if (ctx->cfg.n == 0) return LOSSY_OK;
+  if (ctx->cfg.flags & LOSSY_REPLICA_SKIP_OWNER)
+    return fail(ctx, LOSSY_EINVAL, "closed-loop gradients need every worker's full copy (no LOSSY_REPLICA_SKIP_OWNER)");
   if (!curv || !target || !aligned16(curv) || !aligned16(target)) return fail(ctx, LOSSY_EINVAL, "curv/target: NULL or misaligned");
   if (int rc = check_table(ctx, noise, "noise: NULL or misaligned pointer")) return rc;
-  if (int rc = check_table(ctx, replicas, "replicas: NULL or misaligned pointer")) return rc;
+  if (int rc = check_replicas(ctx, replicas)) return rc;
   if (int rc = check_table(ctx, grads_out, "grads_out: NULL or misaligned pointer")) return rc;
   ClosedLoopArgs A;
   memset(&A, 0, sizeof A);
@@ -818,6 +877,25 @@ int lossy_device_status(lossy_ctx* ctx, void* stream) {
   if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(ctx, "status read", e);
   if (word != 0) return fail(ctx, LOSSY_EDEVICE, "a bounded wait inside a kernel gave up; results of that call are invalid");
+  return LOSSY_OK;
+}
+
+int lossy_reset_status(lossy_ctx* ctx, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  cudaError_t e = cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ticket, 0, sizeof(uint32_t), (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(ctx, "status reset", e);
+  ctx->err[0] = 0;
+  return LOSSY_OK;
+}
+
+int lossy_selftest_wait_expiry(lossy_ctx* ctx, uint32_t max_polls, void* stream) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (max_polls == 0 || max_polls > (1u << 20)) return fail(ctx, LOSSY_EINVAL, "max_polls: 1 .. 2^20");
+  wait_expiry_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(max_polls, ctx->status);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "self-test launch", e);
+  ctx->launches++;
   return LOSSY_OK;
 }
 
@@ -886,6 +964,10 @@ int lossy_mask_grid(lossy_ctx* ctx, uint64_t step, const uint32_t* src, const ui
 
 const char* lossy_last_error(const lossy_ctx* ctx) { return ctx ? ctx->err : "NULL context"; }
 uint64_t lossy_num_packets(const lossy_ctx* ctx) { return ctx ? ctx->K : 0; }
+uint64_t lossy_replica_elems(const lossy_ctx* ctx, uint32_t worker) {
+  if (!ctx || worker >= ctx->cfg.W) return 0;
+  return (ctx->cfg.flags & LOSSY_REPLICA_SKIP_OWNER) ? ctx->cfg.n - own_elems(ctx, worker) : ctx->cfg.n;
+}
 uint64_t lossy_kernel_launches(const lossy_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 int lossy_describe_plan(lossy_ctx* ctx, int with_drift, char* buf, size_t size) {

@@ -25,6 +25,8 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kChunk = 256;  // elements per warp-chunk
 
 enum Phase : int { AGG = 1, STEP = 2, BCAST = 4, DRIFT = 8 };
+// bits of Params::flags that the kernels look at (the values of the public flags of the same meaning)
+constexpr uint32_t kSelfLossless = 1u, kZeroSkip = 2u, kSkipOwner = 8u;
 
 struct Params {
   const void* grads[kMaxW];
@@ -65,7 +67,35 @@ struct Params {
   uint32_t flags;
   uint32_t prefetch_next; // register kernel: L2-prefetch the warp's next chunk
   float lr, b1, b2, omb1, omb2, ibc1, ibc2, eps;
+  // Owner-elided replicas (kSkipOwner): replica i stores this context's elements WITHOUT the packets worker i
+  // owns, so everything behind worker i's shard sits rep_skip[i] elements lower in its array. All zero otherwise.
+  uint64_t rep_skip[kMaxW];
 };
+
+// Owner-elided replicas: rep_skip[i] = elements of worker i's shard inside the context's packet range
+// [k0, k0 + K) of a bucket cut into shards of pps packets (the last packet may be short: n elements in all).
+__host__ inline void fill_rep_skip(Params& P, bool elide) {
+  for (uint32_t i = 0; i < (uint32_t)kMaxW; ++i) P.rep_skip[i] = 0;
+  if (!elide) return;
+  for (uint32_t i = 0; i < P.W; ++i) {
+    const uint64_t s0 = (uint64_t)i * P.pps, s1 = s0 + P.pps;          // shard i in bucket packets
+    const uint64_t c0 = P.k0, c1 = (uint64_t)P.k0 + P.K;                // this context in bucket packets
+    const uint64_t lo = s0 > c0 ? s0 : c0, hi = s1 < c1 ? s1 : c1;
+    if (lo >= hi) continue;
+    const uint64_t e0 = (lo - c0) * P.P, e1 = (hi - c0) * P.P;
+    P.rep_skip[i] = (e1 < P.n ? e1 : P.n) - (e0 < P.n ? e0 : P.n);
+  }
+}
+// Index of bucket element e (in context packet k) inside replica i's array; i must not be k's owner when the
+// replicas are owner-elided.
+__device__ __forceinline__ uint64_t rep_index(const Params& P, uint32_t i, uint32_t k, uint64_t e) {
+  if (!(P.flags & kSkipOwner)) return e;
+  return ((uint64_t)P.k0 + k >= (uint64_t)(i + 1u) * P.pps) ? e - P.rep_skip[i] : e;
+}
+// The replica that does not exist for a packet of owner j (as a bit), or 0 with full replicas.
+__device__ __forceinline__ uint64_t own_bit(const Params& P, uint32_t j) {
+  return (P.flags & kSkipOwner) ? 1ull << j : 0ull;
+}
 
 // ---- delivery-indicator hash (Section 3: s, r ~ Bernoulli(1-p)) -------------
 // 64-bit finalizer of the splitmix64 generator; the constants of the keyed

@@ -239,7 +239,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
             while (sn) {
               const int i = __ffsll((long long)sn) - 1;
               sn &= sn - 1;
-              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + en);
+              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, kn, en));
             }
           }
         }
@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
       while (sm) {
         const int i = __ffsll((long long)sm) - 1;
         sm &= sm - 1;
-        prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e);
+        prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, k, e));
       }
     }
 
@@ -345,13 +345,15 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
       const Vec8<RT> wire = narrow<RT>(th);
       float xw[8];
       widen<RT>(wire, xw);
+      const uint64_t own = own_bit(P, j);   // owner-elided replicas: worker j holds no copy of this packet
       if constexpr (PH & BCAST) {
+        const uint64_t keep = stale | own;
         for (uint32_t i = 0; i < W; ++i)
-          if (!((stale >> i) & 1ull)) store8<RT>(P.replicas[i], e, wire, nvalid);
+          if (!((keep >> i) & 1ull)) store8<RT>(P.replicas[i], rep_index(P, i, k, e), wire, nvalid);
       }
       if constexpr (PH & DRIFT) {
         // copies that differ from the wire value: the stale ones after a broadcast, or (standalone) all
-        uint64_t todo = (PH & BCAST) ? stale : (W == 64 ? ~0ull : ((1ull << W) - 1ull));
+        uint64_t todo = (PH & BCAST) ? stale : ((W == 64 ? ~0ull : ((1ull << W) - 1ull)) & ~own);
         while (todo) {
           // up to four copies are fetched before the first is used
           int ids[4];
@@ -364,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
               ids[b] = __ffsll((long long)todo) - 1;
               todo &= todo - 1;
               nb = b + 1;
-              old[b] = load8_any<RT>(P.replicas[ids[b]], e, nvalid);
+              old[b] = load8_any<RT>(P.replicas[ids[b]], rep_index(P, (uint32_t)ids[b], k, e), nvalid);
             }
           }
 #pragma unroll
@@ -460,6 +462,10 @@ struct PairwiseArgs {
   uint64_t n;
   uint32_t W;
   uint32_t nblk;   // ceil(W / 4)
+  // owner-elided replicas (elide != 0): the owner of an element holds no copy of it, so the element adds only
+  // to the pairs of the other workers; rep_skip as in Params
+  uint32_t elide, P, pps, k0;
+  uint64_t rep_skip[kMaxW];
 };
 
 template <class RT>
@@ -476,17 +482,24 @@ static __global__ void __launch_bounds__(256) drift_pairwise_kernel(const __grid
     const uint64_t e = vi * 8;
     const int nvalid = A.n - e >= 8 ? 8 : (int)(A.n - e);
     float a[4][8], b[4][8];
+    uint32_t owner = 0xFFFFFFFFu;          // the worker without a copy of this vector (a vector lies in one packet)
+    uint64_t kb = 0;                       // its bucket packet
+    if (A.elide) {
+      kb = (uint64_t)A.k0 + e / A.P;
+      owner = (uint32_t)(kb / A.pps);
+    }
+    auto at = [&](uint32_t i) { return (A.elide && kb >= (uint64_t)(i + 1u) * A.pps) ? e - A.rep_skip[i] : e; };
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const uint32_t ia = I * 4 + u, ib = J * 4 + u;
-      if (ia < A.W) widen<RT>(load8_any<RT>(A.replicas[ia], e, nvalid), a[u]);
-      if (ib < A.W) widen<RT>(load8_any<RT>(A.replicas[ib], e, nvalid), b[u]);
+      if (ia < A.W && ia != owner) widen<RT>(load8_any<RT>(A.replicas[ia], at(ia), nvalid), a[u]);
+      if (ib < A.W && ib != owner) widen<RT>(load8_any<RT>(A.replicas[ib], at(ib), nvalid), b[u]);
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
-        if (I * 4 + u < A.W && J * 4 + v < A.W) {
+        if (I * 4 + u < A.W && J * 4 + v < A.W && I * 4 + u != owner && J * 4 + v != owner) {
           float s = 0.0f;
 #pragma unroll
           for (int x = 0; x < 8; ++x) {

@@ -29,6 +29,11 @@ int g_sms[kMaxDevices];
 
 // Set-up, once per device, with that device current: the array's name is only a host-side
 // handle here, so ask the runtime for its device address before giving it to a kernel.
+// This first call on a device is also the one that may load the library's device code (CUDA loads
+// modules lazily), which reserves memory for the kernels and for the array itself: it belongs at
+// start-up, before the caller commits or freezes its memory and before any stream capture. The
+// cached address is valid until the device is reset (cudaDeviceReset); a process that resets a
+// device must not call this entry point on it afterwards.
 int static_scratch(double** out, int* sms) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
@@ -38,6 +43,7 @@ int static_scratch(double** out, int* sms) {
   if (!g_ptr[dev]) {
     double* p = nullptr;
     e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials);
+    if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return LOSSY_ENOMEM; }   // no room left to load the library image
     if (e != cudaSuccess || !p) return LOSSY_ECUDA;
     int n = 0;
     e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
@@ -78,8 +84,14 @@ extern "C" int drift_norms_static(const lossy_config* cfg, const float* master, 
   const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
   const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;
   if (K * cpp > LOSSY_STATIC_MAX_CHUNKS) return LOSSY_ELIMIT;
-  for (uint32_t i = 0; i < cfg->W; ++i)
-    if (!replicas[i] || (reinterpret_cast<uintptr_t>(replicas[i]) & 15u)) return LOSSY_EINVAL;
+  // the shard map (only the owner-elided replica layout depends on it): a packet range of a larger bucket, or the whole bucket
+  const bool elide = (cfg->flags & LOSSY_REPLICA_SKIP_OWNER) != 0;
+  if (cfg->bucket_packets ? (cfg->bucket_packets >= (1ull << 31) || cfg->shard_packet0 + K > cfg->bucket_packets)
+                          : cfg->shard_packet0 != 0)
+    return LOSSY_EINVAL;
+  const uint64_t Kb = cfg->bucket_packets ? cfg->bucket_packets : K;
+  const uint64_t pps = (Kb + cfg->W - 1) / cfg->W;
+
   cudaStream_t s = (cudaStream_t)stream;
   if (cfg->n == 0) {
     if (norms && cudaMemsetAsync(norms, 0, cfg->W * sizeof(float), s) != cudaSuccess) return LOSSY_ECUDA;
@@ -96,10 +108,17 @@ extern "C" int drift_norms_static(const lossy_config* cfg, const float* master, 
   P.n = cfg->n;
   P.num_chunks = (uint32_t)(K * cpp);
   P.chunks_per_packet = (uint32_t)cpp;
-  const uint64_t pps = (K + cfg->W - 1) / cfg->W;
   P.pps = pps ? (uint32_t)pps : 1u;
+  P.k0 = (uint32_t)cfg->shard_packet0;
+  P.K = (uint32_t)K;
   P.P = cfg->packet_elems;
   P.W = cfg->W;
+  P.flags = elide ? kSkipOwner : 0u;
+  fill_rep_skip(P, elide);
+  for (uint32_t i = 0; i < cfg->W; ++i) {
+    if (elide && P.rep_skip[i] == cfg->n) continue;           // this worker owns everything here: its replica holds nothing
+    if (!replicas[i] || (reinterpret_cast<uintptr_t>(replicas[i]) & 15u)) return LOSSY_EINVAL;
+  }
   P.master = const_cast<float*>(master);
   for (uint32_t i = 0; i < cfg->W; ++i) P.replicas[i] = const_cast<void*>(replicas[i]);
   // Every row that the finalize kernel reads is written in full by this call's own blocks

@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         } else if constexpr (PH == STEP) {
           if (P.flags & 2u) cnt = P.count_in[k];
         } else {
-          recv = all;   // standalone drift: every copy is compared
+          recv = all & ~own_bit(P, j);   // standalone drift: every copy that exists is compared
         }
         for (uint32_t g = 0; g < G.groups; ++g) {
           if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
@@ -146,6 +146,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if (lane == 0) {
             StageHdr& h = hdrs[s];
             h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
+            h.own = own_bit(P, j);
             uint32_t bytes = __popc(bits) * len * kEB;
             if constexpr (PH == STEP) bytes = (OPT == 1 ? 4u : 2u) * len * 4u;
             if constexpr (PH == BCAST) bytes = len * 4u;
@@ -156,7 +157,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if constexpr (kGrouped) {
             if (lane < GS && ((bits >> lane) & 1u)) {
               const void* src_p = PH == AGG ? P.grads[g * GS + lane] : P.replicas[g * GS + lane];
-              bulk_g2s(smem_u32(st + (size_t)lane * kTile * kEB), reinterpret_cast<const typename T::raw*>(src_p) + e0,
+              const uint64_t at = PH == AGG ? e0 : rep_index(P, g * GS + (uint32_t)lane, k, e0);
+              bulk_g2s(smem_u32(st + (size_t)lane * kTile * kEB), reinterpret_cast<const typename T::raw*>(src_p) + at,
                        len * kEB, full_bar(s), lh, pol);
             }
             if constexpr (PH == DRIFT) {
@@ -215,10 +217,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             }
           }
         } else if constexpr (PH == BCAST) {
-          const uint64_t stale = h.stale;
+          const uint64_t keep = h.stale | h.own;   // replicas that are not written: they missed the broadcast, or do not exist
           for (uint32_t i = lane; i < W; i += 32)
-            if (!((stale >> i) & 1ull))
-              bulk_s2g(reinterpret_cast<typename T::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kEB, sh_hint, pol);
+            if (!((keep >> i) & 1ull))
+              bulk_s2g(reinterpret_cast<typename T::raw*>(P.replicas[i]) + rep_index(P, i, h.k, e0), smem_u32(st + off_wire), len * kEB,
+                       sh_hint, pol);
         }
         bulk_commit();
         bulk_wait_read0();            // shared memory of this stage may be overwritten after this
@@ -316,11 +319,12 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           }
           // squared differences of this lane's elements against each copy of the group ...
           const uint32_t in_group = min((uint32_t)GS, W - g * GS);
+          const uint32_t have = (uint32_t)(h.recv >> (g * GS)) & ((1u << GS) - 1u);   // the copies that were fetched
           float sq[GS];
 #pragma unroll
           for (int u = 0; u < GS; ++u) {
             sq[u] = 0.0f;
-            if (active && (uint32_t)u < in_group) {
+            if (active && ((have >> u) & 1u)) {
               // two elements per instruction (packed fp32 pairs of sm_100)
               float old[kEpl];
               lds_lane<T>(st + (size_t)u * kTile * kEB, idx, old);

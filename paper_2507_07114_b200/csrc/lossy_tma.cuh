@@ -73,7 +73,8 @@ struct __align__(16) PackedMasks { uint64_t recv[kMaxSub], stale[kMaxSub]; };   
 struct __align__(16) StageHdr {
   uint64_t recv, stale, e0;
   uint32_t k, len, cnt, last;
-  uint32_t pad[6];
+  uint64_t own;          // owner-elided replicas: the bit of the replica that does not exist for this packet
+  uint32_t pad[4];
 };
 static_assert(sizeof(StageHdr) == 64, "header is one 64-byte slot");
 
@@ -134,13 +135,32 @@ __device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Bounded wait; false = gave up (or another role already aborted).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t max_polls = kMaxPolls) {
+  for (uint32_t i = 0; i < max_polls; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1u;
   return false;
+}
+
+// Self-test of the failure report: one small CTA initialises a barrier that nothing ever arms or arrives on,
+// waits on it with the pipelines' own bounded wait (a short poll limit, no copy in flight), and leaves through
+// the pipelines' exit path: abort flag -> the context's status word.
+static __global__ void wait_expiry_kernel(uint32_t max_polls, uint32_t* status) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t abort_word;
+  volatile uint32_t* abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  mbar_wait(smem_u32(&bar), 0u, abort_flag, max_polls);   // phase 0 never completes
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) atomicExch(status, 1u);
 }
 
 // kEpl consecutive elements of one lane, to and from shared or global memory
@@ -302,7 +322,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
           if (lane == 0) {
             StageHdr& h = hdrs[s];
-            h.recv = 0; h.stale = 0; h.e0 = e0; h.k = npk; h.len = len; h.cnt = 0; h.last = last ? 1u : 0u;
+            h.recv = 0; h.stale = 0; h.e0 = e0; h.k = npk; h.len = len; h.cnt = 0; h.last = last ? 1u : 0u; h.own = 0;
             uint32_t bytes = in_group * len * kGB;
             if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
             mbar_arrive_expect_tx(full_bar(s), bytes);
@@ -366,7 +386,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if constexpr (DRIFTK && !kStaleStages) {
             for (uint32_t i = lane; i < W; i += 32)
               if ((stale >> i) & 1ull)
-                bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + e0, len * kRB);
+                bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, k, e0), len * kRB);
           }
           if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
           if constexpr (SPLIT) {
@@ -392,6 +412,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             if (lane == 0) {
               StageHdr& h = hdrs[s];
               h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = g + 1 == G.groups ? 1u : 0u;
+              h.own = own_bit(P, j);
               uint32_t bytes = __popc(bits) * len * kGB;
               if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
               mbar_arrive_expect_tx(full_bar(s), bytes);
@@ -430,13 +451,14 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
               if (lane == 0) {
                 StageHdr& h = hdrs[s];
-                h.recv = ids; h.stale = 0; h.e0 = e0; h.k = k; h.len = len; h.cnt = (uint32_t)__popcll(ids); h.last = 2u;
+                h.recv = ids; h.stale = 0; h.e0 = e0; h.k = k; h.len = len; h.cnt = (uint32_t)__popcll(ids); h.last = 2u; h.own = 0;
                 mbar_arrive_expect_tx(full_bar(s), (uint32_t)__popcll(ids) * len * kRB);
               }
               __syncwarp();
               if (mine >= 0)
                 bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
-                         reinterpret_cast<const typename RT::raw*>(P.replicas[mine]) + e0, len * kRB, full_bar(s), lh, pol);
+                         reinterpret_cast<const typename RT::raw*>(P.replicas[mine]) + rep_index(P, (uint32_t)mine, k, e0), len * kRB,
+                         full_bar(s), lh, pol);
               armed_mask |= 1u << s;
               armed_par = (armed_par & ~(1u << s)) | (par << s);
               if (++s == S) { s = 0; par ^= 1u; }
@@ -471,6 +493,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         if (g + 1 == G.groups) {
           const StageHdr& h = hdrs[s];
           const uint64_t e0 = h.e0, stale = h.stale;
+          const uint64_t keep = stale | h.own;     // replicas that are not written: they missed the broadcast, or do not exist
           const uint32_t len = h.len;
           unsigned char* st = SPLIT ? state0 + (size_t)sq * G.state_bytes : stage0 + (size_t)s * G.stage_bytes;
           if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u, sh_hint, pol);
@@ -487,7 +510,10 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
                 const bool fresh = sp < npk && !((pks[s].stale[sp < npk ? sp : 0] >> i) & 1ull);
                 if (fresh && run < 0) run = (int)sp;
                 if (!fresh && run >= 0) {
-                  bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0 + (uint64_t)run * P.P,
+                  // (with owner-elided replicas a run never holds a packet of worker i's own shard, so one
+                  // index shift serves the whole run)
+                  bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) +
+                               rep_index(P, i, tile * G.packets_per_tile + (uint32_t)run, e0 + (uint64_t)run * P.P),
                            smem_u32(st + off_wire + (size_t)run * P.P * kRB), (sp - (uint32_t)run) * P.P * kRB, sh_hint, pol);
                   run = -1;
                 }
@@ -495,8 +521,9 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             }
           } else {
             for (uint32_t i = lane; i < W; i += 32)
-              if (!((stale >> i) & 1ull))
-                bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + e0, smem_u32(st + off_wire), len * kRB, sh_hint, pol);
+              if (!((keep >> i) & 1ull))
+                bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + rep_index(P, i, h.k, e0), smem_u32(st + off_wire), len * kRB,
+                         sh_hint, pol);
           }
           bulk_commit();
           bulk_wait_read0();          // shared memory of this stage may be overwritten after this
@@ -587,6 +614,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     }
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
       uint64_t my_recv = 0, my_stale = 0;
+      uint32_t my_k = 0;                 // PACKED: the packet this warp's elements lie in
       bool my_first = false;
       if constexpr (PACKED) {
         const uint32_t kfirst = tile * G.packets_per_tile;
@@ -602,6 +630,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           my_first = widx == my_sp * P.P;
           my_recv = tmasks[mbuf].recv[my_sp];
           my_stale = tmasks[mbuf].stale[my_sp];
+          my_k = kfirst + my_sp;
         }
         // the next tile's masks now: their latency hides behind this tile's pipeline waits
         if (tile + gridDim.x < G.num_tiles) eval_masks(tile + gridDim.x, mbuf ^ 1u);
@@ -611,7 +640,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             while (sm) {
               const int i = __ffsll((long long)sm) - 1;
               sm &= sm - 1;
-              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + (uint64_t)kfirst * P.P + idx);
+              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) +
+                          rep_index(P, (uint32_t)i, my_k, (uint64_t)kfirst * P.P + idx));
             }
           }
         }
@@ -653,8 +683,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         }
         const uint32_t cnt = PACKED ? (uint32_t)__popcll(my_recv) : h.cnt;
         const uint64_t stale = PACKED ? my_stale : h.stale, e0 = h.e0;
+        const uint32_t kk = PACKED ? my_k : h.k;      // the packet of this lane's elements
         if constexpr (PACKED) {
-          if (my_first && lane == 0) pks[s].stale[my_sp] = my_stale;   // for the store warp, before this warp's arrive
+          // for the store warp, before this warp's arrive: the replicas that do not take this sub-packet
+          if (my_first && lane == 0)
+            pks[s].stale[my_sp] = my_stale | ((P.flags & kSkipOwner) ? own_bit(P, (P.k0 + my_k) / P.pps) : 0ull);
         }
         float wire[kEpl];
         // The first stale copies are requested now, so that their (L2) latency hides behind the arithmetic
@@ -672,7 +705,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               stale_rest &= stale_rest - 1;
               if (active)
                 load_words_stream<LaneWords<RT>::value>(
-                    reinterpret_cast<const typename RT::raw*>(P.replicas[pre_id[b]]) + e0 + idx, pre_raw[b]);
+                    reinterpret_cast<const typename RT::raw*>(P.replicas[pre_id[b]]) + rep_index(P, (uint32_t)pre_id[b], kk, e0 + idx),
+                    pre_raw[b]);
             }
           }
         }
@@ -817,7 +851,8 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
                 sm &= sm - 1;
                 nb = b + 1;
                 if (active) {
-                  const typename RT::raw* rp = reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) + e0 + idx;
+                  const typename RT::raw* rp =
+                      reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) + rep_index(P, (uint32_t)ids[b], kk, e0 + idx);
                   uint32_t ow[4];
                   load_words_stream<LaneWords<RT>::value>(rp, ow);
                   unpack_lane<RT>(ow, old[b]);

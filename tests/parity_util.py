@@ -63,20 +63,32 @@ class GpuRun:
     """State of one simulated run on the GPU, advanced through the C ABI."""
 
     def __init__(self, w: workload.Workload, *, flags=0, p_grad=None, p_param=None, theta0=None, device="cuda",
-                 alg1=False, burst=None):
+                 alg1=False, burst=None, shard_packet0=0, bucket_packets=0):
         self.w, self.dev, self.alg1, self.burst = w, device, alg1, burst
+        rng_kw = {"shard_packet0": shard_packet0, "bucket_packets": bucket_packets} if bucket_packets else {}
         self.ctx = L.lossy_init(W=w.W, n=w.n, packet_elems=w.packet_elems,
                                 p_grad=w.p if p_grad is None else p_grad,
                                 p_param=w.p if p_param is None else p_param, seed=w.seed,
                                 grad_dtype=tdtype(w.grad_dtype), replica_dtype=tdtype(w.replica_dtype),
                                 optimizer=w.optimizer, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
-                                flags=flags, packet_base=w.packet_base)
+                                flags=flags, packet_base=w.packet_base, **rng_kw)
         n, W, K = w.n, w.W, w.K
         th = workload.theta0_slab(w, 0, n, device) if theta0 is None else theta0.to(device)
         self.master = th.clone()
         self.m = torch.zeros(n, dtype=torch.float32, device=device)
         self.v = torch.zeros(n, dtype=torch.float32, device=device)
-        self.replicas = [self.master.to(tdtype(w.replica_dtype)).clone() for _ in range(W)]
+        self.elided = bool(flags & L.LOSSY_REPLICA_SKIP_OWNER)
+        wire = self.master.to(tdtype(w.replica_dtype))
+        if self.elided:
+            # owner-elided layout: replica i is the bucket without the packets worker i owns
+            Kb = bucket_packets if bucket_packets else K
+            pps = (Kb + W - 1) // W
+            owner = (shard_packet0 + torch.arange(n, device=device) // w.packet_elems) // pps
+            self.replicas = [wire[owner != i].clone() for i in range(W)]
+            for i in range(W):
+                assert self.replicas[i].numel() == L.lossy_replica_elems(self.ctx, i)
+        else:
+            self.replicas = [wire.clone() for _ in range(W)]
         self.ghat = torch.zeros(n, dtype=torch.float32, device=device)
         self.ghat_prev = torch.zeros(n, dtype=torch.float32, device=device) if alg1 else None
         self.count = torch.zeros(K, dtype=torch.uint8, device=device)
@@ -151,13 +163,26 @@ def make_oracle(w: workload.Workload, *, flags=0, p_grad=None, p_param=None, the
 
 
 def compare_state(gpu: GpuRun, orc, what, e0=0, e1=None):
+    whole = e0 == 0 and e1 is None
     e1 = gpu.w.n if e1 is None else e1
     assert_rel(to_np(gpu.master[e0:e1]), orc.master, f"{what} master")
     if gpu.w.optimizer == "adam":
         assert_rel(to_np(gpu.m[e0:e1]), orc.m, f"{what} m")
         assert_rel(to_np(gpu.v[e0:e1]), orc.v, f"{what} v")
     for i in range(gpu.w.W):
-        assert_rel(to_np(gpu.replicas[i][e0:e1]), orc.replicas[i], f"{what} replica {i}")
+        if gpu.elided and not whole:
+            # a slab [e0, e1) of an owner-elided replica: the slab's elements that worker i does not own, which
+            # start where the elements in front of the slab that it does not own end
+            P, K = gpu.w.packet_elems, gpu.w.K
+            pps = (K + gpu.w.W - 1) // gpu.w.W
+            lo, hi = min(gpu.w.n, i * pps * P), min(gpu.w.n, (i + 1) * pps * P)      # worker i's own elements
+            own_before = max(0, min(hi, e0) - lo)
+            own_inside = max(0, min(hi, e1) - max(lo, e0))
+            a = e0 - own_before
+            got = gpu.replicas[i][a:a + (e1 - e0) - own_inside]
+        else:
+            got = gpu.replicas[i] if gpu.elided else gpu.replicas[i][e0:e1]
+        assert_rel(to_np(got), orc.replicas[i], f"{what} replica {i}")
 
 
 def compare_outputs(out, ref, what, with_ghat=True):
@@ -174,7 +199,7 @@ def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None,
                alg1=False, burst=None):
     """Element-by-element parity of a whole (small) run. Returns the GpuRun for further checks."""
     gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param, alg1=alg1, burst=burst)
-    orc = make_oracle(w, flags=flags & 3, p_grad=p_grad, p_param=p_param, alg1=alg1, burst=burst)   # bit 4 only picks the kernel
+    orc = make_oracle(w, flags=flags & ~L.LOSSY_REGISTER_PATH, p_grad=p_grad, p_param=p_param, alg1=alg1, burst=burst)   # that bit only picks the kernel
     for t in range(1, steps + 1):
         gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]
         gd = [g.cuda() for g in gs]

@@ -191,7 +191,7 @@ def test_empty_bucket_is_a_noop_and_bad_arguments_are_rejected():
     assert L.lossy_kernel_launches(ctx) == 0
     L.lossy_destroy(ctx)
     for bad in (dict(W=0), dict(W=65), dict(packet_elems=0), dict(packet_elems=12), dict(p_grad=1.0),
-                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=8), dict(optimizer=5)):
+                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=16), dict(optimizer=5)):
         kw = dict(W=2, n=64, packet_elems=64, p_grad=0.1, p_param=0.1, seed=0, grad_dtype=torch.float32,
                   replica_dtype=torch.float32, optimizer="sgd", lr=0.1)
         kw.update(bad)
@@ -331,3 +331,28 @@ def test_launch_policy_picks_the_expected_build_for_the_benchmark_configurations
     assert plan(64, 4096, 0.3)[1] == "bulk-copy twin group=8 stale=late split stages=4"   # no drift norms asked for
     assert plan(8, 2048, 0.1, flags=L.LOSSY_REGISTER_PATH)[0] == "register kernel"
     assert plan(8, 2048, 0.1, n=1000)[0] == "register kernel"                             # no complete packet
+
+
+def test_packed_build_many_tiles_per_cta_with_skewed_stale_sets():
+    """The PACKED build shares a tile's masks between its compute warps through two alternating buffers.
+    Many tiles per CTA (forty) and sub-packets whose stale sets differ wildly (every fourth packet of a tile
+    has a reliable broadcast, the others lose most of theirs) let the warps of a CTA drift far apart; the
+    whole state must still match the oracle element by element."""
+    W, P = 8, 256
+    n = 2048 * 148 * 40 + 256 * 3
+    w = workload.Workload("packed_skew", W, n, P, 0.0, "adam", 3e-4, "bf16", "bf16", 4, seed=77)
+    gpu = GpuRun(w, p_grad=0.2, p_param=0.7)
+    assert "packed" in L.lossy_describe_plan(gpu.ctx)
+    orc = make_oracle(w, p_grad=0.2, p_param=0.7)
+    K = w.K
+    rel = np.zeros((2, K), np.uint64)
+    rel[1, ::4] = np.uint64((1 << W) - 1)                 # these broadcasts always arrive
+    rel_d = torch.from_numpy(rel.view(np.int64)).cuda()
+    L.lossy_set_reliable(gpu.ctx, rel_d)
+    for t in range(1, 4):
+        gs = [workload.grad_slab(w, t, i, 0, n, "cuda") for i in range(W)]
+        gpu.step_fused(t, gs)
+        ref = orc.step(t, [to_np(g) for g in gs], reliable=rel)
+        compare_outputs(gpu.outputs(), ref, f"packed skew step {t}")
+        compare_state(gpu, orc, f"packed skew step {t}")
+    L.lossy_device_status(gpu.ctx)

@@ -12,7 +12,7 @@ import torch
 
 import paper_2507_07114_b200 as L
 import workload
-from parity_util import GpuRun, REL_TOL
+from parity_util import GpuRun, REL_TOL, make_oracle, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -40,6 +40,12 @@ def test_static_scratch_variant_matches_drift_norms_on_two_calls_in_a_row(rdt, W
         assert float(want.max()) > 0.0
         assert _rel(got, want) <= REL_TOL
         assert _rel(got_sq, want_sq) <= 2 * REL_TOL
+        # and against the CPU oracle's own drift routine, run on the state the GPU holds
+        orc = make_oracle(w)
+        orc.master, orc.replicas = to_np(run.master), [to_np(r) for r in run.replicas]
+        ref_sq = torch.from_numpy(orc.drift_sumsq())
+        assert _rel(got_sq, ref_sq) <= 2 * REL_TOL
+        assert _rel(got, ref_sq.sqrt()) <= REL_TOL
     # sumsq is added to, norms alone is allowed
     L.drift_norms_static(W=W, n=n, packet_elems=P, replica_dtype=run.replicas[0].dtype, master=run.master,
                          replicas=run.replicas, sumsq=got_sq)
