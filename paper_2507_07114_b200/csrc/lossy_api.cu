@@ -121,7 +121,7 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
 }
 
 // ---- bulk-copy pipeline (fused step only) --------------------------------------------------
-constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)) + 2 * sizeof(PackedMasks);
+constexpr uint32_t kTmaSmemFixed = kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)) + kMaskBufs * sizeof(PackedMasks);
 
 // Launch policy of the bulk-copy pipeline, from sweeps on B200 over W = 2..64, p = 0.05..0.3
 // (CUDA-event timings of bench.py with each build forced): which of the four builds runs and whether its bulk copies carry an
@@ -331,9 +331,9 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
                          : try_tma<8, 8>(ctx, P, drift, s, blocks, used);
 }
 
-template <int PH, class GT, class RT, int OPT>
+template <int PH, class GT, class RT, int OPT, bool ELIDE = false>
 int launch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_kernel<PH, GT, RT, OPT>;
+  auto kern = lossy_kernel<PH, GT, RT, OPT, ELIDE>;
   static int occupancy[kMaxDevices];   // per kernel instantiation and device: resident blocks per SM
   int per_sm = 0;
   cudaError_t e;
@@ -373,8 +373,16 @@ int dispatch(lossy_ctx* ctx, const Params& P, cudaStream_t s, uint32_t* blocks) 
   } else if constexpr (PH == STEP) {
     return adam ? launch<PH, F32, F32, 1>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
   } else if constexpr (PH == BCAST || PH == DRIFT) {
+    if (ctx->cfg.flags & LOSSY_REPLICA_SKIP_OWNER)   // owner-elided replicas: builds of their own
+      return rb ? launch<PH, F32, BF16, 0, true>(ctx, P, s, blocks) : launch<PH, F32, F32, 0, true>(ctx, P, s, blocks);
     return rb ? launch<PH, F32, BF16, 0>(ctx, P, s, blocks) : launch<PH, F32, F32, 0>(ctx, P, s, blocks);
   } else {
+    if (ctx->cfg.flags & LOSSY_REPLICA_SKIP_OWNER) {
+      if (gb && rb) return adam ? launch<PH, BF16, BF16, 1, true>(ctx, P, s, blocks) : launch<PH, BF16, BF16, 0, true>(ctx, P, s, blocks);
+      if (gb && !rb) return adam ? launch<PH, BF16, F32, 1, true>(ctx, P, s, blocks) : launch<PH, BF16, F32, 0, true>(ctx, P, s, blocks);
+      if (!gb && rb) return adam ? launch<PH, F32, BF16, 1, true>(ctx, P, s, blocks) : launch<PH, F32, BF16, 0, true>(ctx, P, s, blocks);
+      return adam ? launch<PH, F32, F32, 1, true>(ctx, P, s, blocks) : launch<PH, F32, F32, 0, true>(ctx, P, s, blocks);
+    }
     if (gb && rb) return adam ? launch<PH, BF16, BF16, 1>(ctx, P, s, blocks) : launch<PH, BF16, BF16, 0>(ctx, P, s, blocks);
     if (gb && !rb) return adam ? launch<PH, BF16, F32, 1>(ctx, P, s, blocks) : launch<PH, BF16, F32, 0>(ctx, P, s, blocks);
     if (!gb && rb) return adam ? launch<PH, F32, BF16, 1>(ctx, P, s, blocks) : launch<PH, F32, BF16, 0>(ctx, P, s, blocks);

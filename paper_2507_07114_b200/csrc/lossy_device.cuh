@@ -86,11 +86,10 @@ __host__ inline void fill_rep_skip(Params& P, bool elide) {
     P.rep_skip[i] = (e1 < P.n ? e1 : P.n) - (e0 < P.n ? e0 : P.n);
   }
 }
-// Index of bucket element e (in context packet k) inside replica i's array; i must not be k's owner when the
-// replicas are owner-elided.
-__device__ __forceinline__ uint64_t rep_index(const Params& P, uint32_t i, uint32_t k, uint64_t e) {
-  if (!(P.flags & kSkipOwner)) return e;
-  return ((uint64_t)P.k0 + k >= (uint64_t)(i + 1u) * P.pps) ? e - P.rep_skip[i] : e;
+// Index of bucket element e, which lies in a packet owned by worker j, inside replica i's array (i != j when
+// the replicas are owner-elided; with full replicas every rep_skip is 0 and the index is e).
+__device__ __forceinline__ uint64_t rep_index(const Params& P, uint32_t i, uint32_t j, uint64_t e) {
+  return e - (j > i ? P.rep_skip[i] : 0ull);
 }
 // The replica that does not exist for a packet of owner j (as a bit), or 0 with full replicas.
 __device__ __forceinline__ uint64_t own_bit(const Params& P, uint32_t j) {

@@ -191,8 +191,11 @@ __device__ __forceinline__ void batch_masks(const Params& P, const BatchDraws& d
   }
 }
 
-template <int PH, class GT, class RT, int OPT>
+// ELIDE = owner-elided replicas: a build of its own, so that the index arithmetic of that layout costs the
+// default layout nothing (this kernel is bound by its issue slots, not by memory).
+template <int PH, class GT, class RT, int OPT, bool ELIDE = false>
 __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const __grid_constant__ Params P) {
+  auto rep_at = [&](uint32_t i, uint32_t j, uint64_t e) { return ELIDE ? rep_index(P, i, j, e) : e; };
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const uint32_t W = P.W;
@@ -239,7 +242,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
             while (sn) {
               const int i = __ffsll((long long)sn) - 1;
               sn &= sn - 1;
-              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, kn, en));
+              prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_at(i, (P.k0 + kn) / P.pps, en));
             }
           }
         }
@@ -268,7 +271,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
       while (sm) {
         const int i = __ffsll((long long)sm) - 1;
         sm &= sm - 1;
-        prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, k, e));
+        prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_at(i, j, e));
       }
     }
 
@@ -345,11 +348,11 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
       const Vec8<RT> wire = narrow<RT>(th);
       float xw[8];
       widen<RT>(wire, xw);
-      const uint64_t own = own_bit(P, j);   // owner-elided replicas: worker j holds no copy of this packet
+      const uint64_t own = ELIDE ? 1ull << j : 0ull;   // owner-elided replicas: worker j holds no copy of this packet
       if constexpr (PH & BCAST) {
         const uint64_t keep = stale | own;
         for (uint32_t i = 0; i < W; ++i)
-          if (!((keep >> i) & 1ull)) store8<RT>(P.replicas[i], rep_index(P, i, k, e), wire, nvalid);
+          if (!((keep >> i) & 1ull)) store8<RT>(P.replicas[i], rep_at(i, j, e), wire, nvalid);
       }
       if constexpr (PH & DRIFT) {
         // copies that differ from the wire value: the stale ones after a broadcast, or (standalone) all
@@ -366,7 +369,7 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
               ids[b] = __ffsll((long long)todo) - 1;
               todo &= todo - 1;
               nb = b + 1;
-              old[b] = load8_any<RT>(P.replicas[ids[b]], rep_index(P, (uint32_t)ids[b], k, e), nvalid);
+              old[b] = load8_any<RT>(P.replicas[ids[b]], rep_at((uint32_t)ids[b], j, e), nvalid);
             }
           }
 #pragma unroll

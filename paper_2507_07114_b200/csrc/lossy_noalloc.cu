@@ -56,9 +56,9 @@ int static_scratch(double** out, int* sms) {
   return LOSSY_OK;
 }
 
-template <class RT>
+template <class RT, bool ELIDE>
 int launch_static(const Params& P, int sms, cudaStream_t s, uint32_t* blocks_out) {
-  auto kern = lossy_kernel<DRIFT, F32, RT, 0>;
+  auto kern = lossy_kernel<DRIFT, F32, RT, 0, ELIDE>;
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kThreads, 0) != cudaSuccess) return LOSSY_ECUDA;
   if (per_sm < 1) per_sm = 1;
@@ -125,7 +125,9 @@ extern "C" int drift_norms_static(const lossy_config* cfg, const float* master, 
   // first, so nothing in the shared array has to start at zero.
   P.partials = scratch;
   uint32_t blocks = 0;
-  int rc = cfg->replica_dtype == LOSSY_BF16 ? launch_static<BF16>(P, sms, s, &blocks) : launch_static<F32>(P, sms, s, &blocks);
+  int rc;
+  if (elide) rc = cfg->replica_dtype == LOSSY_BF16 ? launch_static<BF16, true>(P, sms, s, &blocks) : launch_static<F32, true>(P, sms, s, &blocks);
+  else rc = cfg->replica_dtype == LOSSY_BF16 ? launch_static<BF16, false>(P, sms, s, &blocks) : launch_static<F32, false>(P, sms, s, &blocks);
   if (rc) return rc;
   drift_finalize_kernel<<<cfg->W, 32, 0, s>>>(scratch, blocks, cfg->W, norms, sumsq);
   return cudaGetLastError() == cudaSuccess ? LOSSY_OK : LOSSY_ECUDA;

@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if (lane == 0) {
             StageHdr& h = hdrs[s];
             h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = last ? 1u : 0u;
-            h.own = own_bit(P, j);
+            h.own = own_bit(P, j); h.j = j;
             uint32_t bytes = __popc(bits) * len * kEB;
             if constexpr (PH == STEP) bytes = (OPT == 1 ? 4u : 2u) * len * 4u;
             if constexpr (PH == BCAST) bytes = len * 4u;
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if constexpr (kGrouped) {
             if (lane < GS && ((bits >> lane) & 1u)) {
               const void* src_p = PH == AGG ? P.grads[g * GS + lane] : P.replicas[g * GS + lane];
-              const uint64_t at = PH == AGG ? e0 : rep_index(P, g * GS + (uint32_t)lane, k, e0);
+              const uint64_t at = PH == AGG ? e0 : rep_index(P, g * GS + (uint32_t)lane, j, e0);
               bulk_g2s(smem_u32(st + (size_t)lane * kTile * kEB), reinterpret_cast<const typename T::raw*>(src_p) + at,
                        len * kEB, full_bar(s), lh, pol);
             }
@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           const uint64_t keep = h.stale | h.own;   // replicas that are not written: they missed the broadcast, or do not exist
           for (uint32_t i = lane; i < W; i += 32)
             if (!((keep >> i) & 1ull))
-              bulk_s2g(reinterpret_cast<typename T::raw*>(P.replicas[i]) + rep_index(P, i, h.k, e0), smem_u32(st + off_wire), len * kEB,
+              bulk_s2g(reinterpret_cast<typename T::raw*>(P.replicas[i]) + rep_index(P, i, h.j, e0), smem_u32(st + off_wire), len * kEB,
                        sh_hint, pol);
         }
         bulk_commit();

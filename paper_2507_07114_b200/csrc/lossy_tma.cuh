@@ -41,8 +41,14 @@ template <int CW> struct TmaShape {
 };
 constexpr int kStaleBatch = 4;                            // stale replica packets in flight per compute lane (8 measured slower)
 constexpr int kMaxStages = 4;                             // deeper pipelines measured no faster
-constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 per stage, 4 of the state slots, 2 of the PACKED masks; 8 B each) and the abort flag
-static_assert((3 * kMaxStages + 6) * 8 + 4 <= (int)kTmaBarBytes, "barrier area too small");
+// PACKED builds: a tile's masks are evaluated one tile ahead and shared through a ring of kMaskBufs buffers.
+// Per warp and iteration n the order is write(n+1), arrive(n+1), wait(n), read(n). A warp that has passed
+// wait(n-1) knows that every warp has arrived for tile n-1, i.e. has entered iteration n-2 and so has finished
+// read(n-3): tile n+1 may therefore reuse the buffer of tile n-3, and no earlier one. Hence four buffers (with
+// two, a warp that is ahead overwrites masks a slower warp has yet to read).
+constexpr uint32_t kMaskBufs = 4;
+constexpr uint32_t kTmaBarBytes = 256;                   // barriers (3 per stage, 4 of the state slots, kMaskBufs of the PACKED masks; 8 B each) and the abort flag
+static_assert((3 * kMaxStages + 4 + kMaskBufs) * 8 + 4 <= kTmaBarBytes, "barrier area too small");
 constexpr uint32_t kMaxPolls = 1u << 22;
 
 struct TmaGeom {
@@ -67,14 +73,15 @@ struct TmaGeom {
 // elements lie in one sub-packet, whose masks it reads from there. The store warp writes each replica the
 // runs of consecutive sub-packets whose broadcast it received.
 constexpr int kMaxSub = 8;
-struct __align__(16) PackedStale { uint64_t stale[kMaxSub]; };
-struct __align__(16) PackedMasks { uint64_t recv[kMaxSub], stale[kMaxSub]; };   // a tile's masks, shared by its compute warps
+struct __align__(16) PackedStale { uint64_t stale[kMaxSub]; uint32_t j[kMaxSub]; };   // per sub-packet: replicas not written, owner
+struct __align__(16) PackedMasks { uint64_t recv[kMaxSub], stale[kMaxSub]; uint32_t j[kMaxSub]; };   // a tile's masks and owners, shared by its compute warps
 
 struct __align__(16) StageHdr {
   uint64_t recv, stale, e0;
   uint32_t k, len, cnt, last;
   uint64_t own;          // owner-elided replicas: the bit of the replica that does not exist for this packet
-  uint32_t pad[4];
+  uint32_t j;            // owner of the packet
+  uint32_t pad[3];
 };
 static_assert(sizeof(StageHdr) == 64, "header is one 64-byte slot");
 
@@ -249,14 +256,14 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
   static_assert(!(SPLIT && PACKED), "the PACKED builds keep the state in the stage");
   static_assert(!kStaleStages || (sizeof(typename RT::raw) <= sizeof(typename GT::raw) && GS == 8), "stale stages reuse the gradient slots");
   // layout: [full, done, empty barriers | abort flag] (kTmaBarBytes) | headers (kMaxStages x 64 B) |
-  //         stale masks per sub-packet of the PACKED build (kMaxStages x 64 B) | two tiles' masks of the PACKED
-  //         build (2 x 128 B) | stages
+  //         stale masks and owners per sub-packet of the PACKED build (one per stage) | the ring of tile masks of
+  //         the PACKED build (kMaskBufs) | stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
   volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kTmaBarBytes - 4);
   StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + kTmaBarBytes);
   PackedStale* pks = reinterpret_cast<PackedStale*>(smem + kTmaBarBytes + kMaxStages * sizeof(StageHdr));
-  PackedMasks* tmasks = reinterpret_cast<PackedMasks*>(smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)));   // [2]
-  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)) + 2 * sizeof(PackedMasks);
+  PackedMasks* tmasks = reinterpret_cast<PackedMasks*>(smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)));   // [kMaskBufs]
+  unsigned char* stage0 = smem + kTmaBarBytes + kMaxStages * (sizeof(StageHdr) + sizeof(PackedStale)) + kMaskBufs * sizeof(PackedMasks);
   const uint32_t S = G.stages;
   // SPLIT builds: two state slots behind the stages
   unsigned char* state0 = stage0 + (size_t)S * G.stage_bytes;
@@ -292,7 +299,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       }
     }
     if constexpr (PACKED) {
-      for (uint32_t q = 0; q < 2; ++q) mbar_init(mask_bar(q), kConsumerWarps);
+      for (uint32_t q = 0; q < kMaskBufs; ++q) mbar_init(mask_bar(q), kConsumerWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -322,7 +329,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
           if (lane == 0) {
             StageHdr& h = hdrs[s];
-            h.recv = 0; h.stale = 0; h.e0 = e0; h.k = npk; h.len = len; h.cnt = 0; h.last = last ? 1u : 0u; h.own = 0;
+            h.recv = 0; h.stale = 0; h.e0 = e0; h.k = npk; h.len = len; h.cnt = 0; h.last = last ? 1u : 0u; h.own = 0; h.j = 0;
             uint32_t bytes = in_group * len * kGB;
             if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
             mbar_arrive_expect_tx(full_bar(s), bytes);
@@ -386,7 +393,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           if constexpr (DRIFTK && !kStaleStages) {
             for (uint32_t i = lane; i < W; i += 32)
               if ((stale >> i) & 1ull)
-                bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, k, e0), len * kRB);
+                bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, j, e0), len * kRB);
           }
           if (P.ghat_prev && cnt == 0 && lane == 0) bulk_prefetch_l2(P.ghat_prev + e0, len * 4u);   // Algorithm 1 fallback
           if constexpr (SPLIT) {
@@ -412,7 +419,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
             if (lane == 0) {
               StageHdr& h = hdrs[s];
               h.recv = recv; h.stale = stale; h.e0 = e0; h.k = k; h.len = len; h.cnt = cnt; h.last = g + 1 == G.groups ? 1u : 0u;
-              h.own = own_bit(P, j);
+              h.own = own_bit(P, j); h.j = j;
               uint32_t bytes = __popc(bits) * len * kGB;
               if (last) bytes += (OPT == 1 ? 3u : 1u) * len * 4u;
               mbar_arrive_expect_tx(full_bar(s), bytes);
@@ -451,13 +458,13 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
               if (lane == 0) {
                 StageHdr& h = hdrs[s];
-                h.recv = ids; h.stale = 0; h.e0 = e0; h.k = k; h.len = len; h.cnt = (uint32_t)__popcll(ids); h.last = 2u; h.own = 0;
+                h.recv = ids; h.stale = 0; h.e0 = e0; h.k = k; h.len = len; h.cnt = (uint32_t)__popcll(ids); h.last = 2u; h.own = 0; h.j = j;
                 mbar_arrive_expect_tx(full_bar(s), (uint32_t)__popcll(ids) * len * kRB);
               }
               __syncwarp();
               if (mine >= 0)
                 bulk_g2s(smem_u32(st + (size_t)lane * kTile * kGB),
-                         reinterpret_cast<const typename RT::raw*>(P.replicas[mine]) + rep_index(P, (uint32_t)mine, k, e0), len * kRB,
+                         reinterpret_cast<const typename RT::raw*>(P.replicas[mine]) + rep_index(P, (uint32_t)mine, j, e0), len * kRB,
                          full_bar(s), lh, pol);
               armed_mask |= 1u << s;
               armed_par = (armed_par & ~(1u << s)) | (par << s);
@@ -513,7 +520,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
                   // (with owner-elided replicas a run never holds a packet of worker i's own shard, so one
                   // index shift serves the whole run)
                   bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) +
-                               rep_index(P, i, tile * G.packets_per_tile + (uint32_t)run, e0 + (uint64_t)run * P.P),
+                               rep_index(P, i, pks[s].j[run], e0 + (uint64_t)run * P.P),
                            smem_u32(st + off_wire + (size_t)run * P.P * kRB), (sp - (uint32_t)run) * P.P * kRB, sh_hint, pol);
                   run = -1;
                 }
@@ -522,7 +529,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           } else {
             for (uint32_t i = lane; i < W; i += 32)
               if (!((keep >> i) & 1ull))
-                bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + rep_index(P, i, h.k, e0), smem_u32(st + off_wire), len * kRB,
+                bulk_s2g(reinterpret_cast<typename RT::raw*>(P.replicas[i]) + rep_index(P, i, h.j, e0), smem_u32(st + off_wire), len * kRB,
                          sh_hint, pol);
           }
           bulk_commit();
@@ -567,9 +574,9 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     // lengthening one warp's tile (with W <= 4 a single pass could cover all eight, and did so at a loss)
     const uint32_t pk_Bp = min(32u >> pk_lgWp, 2u);
     const uint32_t pk_wmask = pk_Wp == 32 ? 0xFFFFFFFFu : ((1u << pk_Wp) - 1u);
-    // PACKED: a tile's masks are evaluated once, one tile ahead, and shared through two alternating buffers
-    // (the main loop reads a tile's masks before it writes the next tile's, which is what keeps a warp that
-    // is ahead from overwriting masks still to be read): with W <= 32 (not Algorithm 1) warp w
+    // PACKED: a tile's masks are evaluated once, one tile ahead, and shared through the ring of kMaskBufs
+    // buffers (see there for why a warp that is ahead never overwrites masks still to be read): with W <= 32
+    // (not Algorithm 1) warp w
     // takes the w-th batch of 32 / Wp sub-packets in one pass of draws; otherwise the first warp of each
     // sub-packet takes its own. Every compute warp arrives on the buffer's barrier once per tile.
     auto eval_masks = [&](uint32_t tile, uint32_t buf) {
@@ -577,10 +584,11 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
       const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
       const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;
       PackedMasks& tm = tmasks[buf];
-      auto report = [&](uint32_t sp, uint64_t r, uint64_t st, uint64_t gbad, uint64_t pbad) {   // one lane
+      auto report = [&](uint32_t sp, uint32_t j, uint64_t r, uint64_t st, uint64_t gbad, uint64_t pbad) {   // one lane
         const uint32_t k = kfirst + sp;
         tm.recv[sp] = r;
         tm.stale[sp] = st;
+        tm.j[sp] = j;
         if (P.count) P.count[k] = (uint8_t)__popcll(r);
         if (P.recv_bits) P.recv_bits[k] = r;
         if (P.stale_bits) P.stale_bits[k] = st;
@@ -594,17 +602,20 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         if (q0 < npk) {
           const uint32_t sp_l = q0 + ((uint32_t)lane >> pk_lgWp), i_l = (uint32_t)lane & (pk_Wp - 1u);
           const uint32_t k_l = kfirst + (sp_l < npk ? sp_l : 0u);
-          const BatchDraws d = batch_draws<AGG | BCAST>(P, k_l, (P.k0 + k_l) / P.pps, i_l, sp_l < npk && i_l < W);
+          const uint32_t j_l = (P.k0 + k_l) / P.pps;
+          const BatchDraws d = batch_draws<AGG | BCAST>(P, k_l, j_l, i_l, sp_l < npk && i_l < W);
           for (uint32_t x = 0; x < pk_Bp && q0 + x < npk; ++x) {
             uint64_t r, st, gbad, pbad;
             batch_masks<AGG | BCAST>(P, d, kfirst + q0 + x, (int)(x * pk_Wp), pk_wmask, r, st, gbad, pbad);
-            if ((uint32_t)lane == x) report(q0 + x, r, st, gbad, pbad);
+            const uint32_t j_x = __shfl_sync(0xFFFFFFFFu, j_l, (int)(x * pk_Wp));   // the owner of sub-packet q0 + x
+            if ((uint32_t)lane == x) report(q0 + x, j_x, r, st, gbad, pbad);
           }
         }
       } else if (widx < npk * P.P && widx == my_sp * P.P) {
         uint64_t r, st, gbad, pbad;
-        packet_masks<AGG | BCAST>(P, kfirst + my_sp, (P.k0 + kfirst + my_sp) / P.pps, lane, r, st, gbad, pbad);
-        if (lane == 0) report(my_sp, r, st, gbad, pbad);
+        const uint32_t j_sp = (P.k0 + kfirst + my_sp) / P.pps;
+        packet_masks<AGG | BCAST>(P, kfirst + my_sp, j_sp, lane, r, st, gbad, pbad);
+        if (lane == 0) report(my_sp, j_sp, r, st, gbad, pbad);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(mask_bar(buf));
@@ -614,38 +625,32 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
     }
     for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
       uint64_t my_recv = 0, my_stale = 0;
-      uint32_t my_k = 0;                 // PACKED: the packet this warp's elements lie in
+      uint32_t my_j = 0;                 // PACKED: the owner of the packet this warp's elements lie in
       bool my_first = false;
       if constexpr (PACKED) {
         const uint32_t kfirst = tile * G.packets_per_tile;
         const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
         const uint32_t widx = (uint32_t)(threadIdx.x & ~31) * kEpl;
-        // This tile's masks (written one iteration ago) are copied to registers BEFORE the next tile's are
-        // written into the other buffer. Order of events per warp and iteration n: wait(n), read(n), write(n+1),
-        // arrive(n+1). A warp's wait(n) therefore proves that every warp has arrived for tile n, i.e. has
-        // finished read(n-1) — so write(n+1), which reuses the buffer of tile n-1, overwrites nothing that is
-        // still to be read, however far the warps of a CTA drift apart inside a tile.
+        // the next tile's masks first (their latency hides behind the wait for this tile's), into the buffer
+        // three behind this tile's
+        if (tile + gridDim.x < G.num_tiles) eval_masks(tile + gridDim.x, (mbuf + 1u) & (kMaskBufs - 1u));
         if (!mbar_wait(mask_bar(mbuf), mpar, abort_flag)) { ok = false; break; }
         if (widx < npk * P.P) {
           my_first = widx == my_sp * P.P;
           my_recv = tmasks[mbuf].recv[my_sp];
           my_stale = tmasks[mbuf].stale[my_sp];
-          my_k = kfirst + my_sp;
-        }
-        // the next tile's masks now: their latency hides behind this tile's pipeline waits
-        if (tile + gridDim.x < G.num_tiles) eval_masks(tile + gridDim.x, mbuf ^ 1u);
-        if (widx < npk * P.P) {
-          if constexpr (DRIFTK) {
+          my_j = tmasks[mbuf].j[my_sp];
+          if constexpr (DRIFTK) {   // the old copies this warp will compare against: start them toward L2 right away
             uint64_t sm = my_stale;
             while (sm) {
               const int i = __ffsll((long long)sm) - 1;
               sm &= sm - 1;
               prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) +
-                          rep_index(P, (uint32_t)i, my_k, (uint64_t)kfirst * P.P + idx));
+                          rep_index(P, (uint32_t)i, my_j, (uint64_t)kfirst * P.P + idx));
             }
           }
         }
-        if (++mbuf == 2u) { mbuf = 0; mpar ^= 1u; }
+        if (++mbuf == kMaskBufs) { mbuf = 0; mpar ^= 1u; }
       }
       for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
         if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
@@ -683,11 +688,13 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         }
         const uint32_t cnt = PACKED ? (uint32_t)__popcll(my_recv) : h.cnt;
         const uint64_t stale = PACKED ? my_stale : h.stale, e0 = h.e0;
-        const uint32_t kk = PACKED ? my_k : h.k;      // the packet of this lane's elements
+        const uint32_t jj = PACKED ? my_j : h.j;      // the owner of the packet of this lane's elements
         if constexpr (PACKED) {
           // for the store warp, before this warp's arrive: the replicas that do not take this sub-packet
-          if (my_first && lane == 0)
-            pks[s].stale[my_sp] = my_stale | ((P.flags & kSkipOwner) ? own_bit(P, (P.k0 + my_k) / P.pps) : 0ull);
+          if (my_first && lane == 0) {
+            pks[s].stale[my_sp] = my_stale | own_bit(P, my_j);
+            pks[s].j[my_sp] = my_j;
+          }
         }
         float wire[kEpl];
         // The first stale copies are requested now, so that their (L2) latency hides behind the arithmetic
@@ -705,7 +712,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
               stale_rest &= stale_rest - 1;
               if (active)
                 load_words_stream<LaneWords<RT>::value>(
-                    reinterpret_cast<const typename RT::raw*>(P.replicas[pre_id[b]]) + rep_index(P, (uint32_t)pre_id[b], kk, e0 + idx),
+                    reinterpret_cast<const typename RT::raw*>(P.replicas[pre_id[b]]) + rep_index(P, (uint32_t)pre_id[b], jj, e0 + idx),
                     pre_raw[b]);
             }
           }
@@ -852,7 +859,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
                 nb = b + 1;
                 if (active) {
                   const typename RT::raw* rp =
-                      reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) + rep_index(P, (uint32_t)ids[b], kk, e0 + idx);
+                      reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) + rep_index(P, (uint32_t)ids[b], jj, e0 + idx);
                   uint32_t ow[4];
                   load_words_stream<LaneWords<RT>::value>(rp, ow);
                   unpack_lane<RT>(ow, old[b]);

@@ -41,7 +41,7 @@ def test_closed_loop_matches_the_oracle(case):
 
 
 def test_objective_degrades_gently_with_the_drop_rate():
-    from paper_2507_07114_b200.closed_loop import run
+    from bench import closed_loop_run as run
 
     vals = [run(p, W=8, n=2048 * 512, P=2048, steps=120, optimizer="sgd", lr=0.1, gdt=torch.float32,
                 rdt=torch.float32)[0] for p in (0.0, 0.1, 0.3)]
