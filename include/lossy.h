@@ -83,7 +83,11 @@ enum {
    * fits one 180 GB GPU). A replica that would hold nothing (W = 1) may be NULL.
    * drift_pairwise then sums, on every element, over the pairs of workers that both hold a copy;
    * lossy_closed_loop_grads needs full replicas and rejects such a context. */
-  LOSSY_REPLICA_SKIP_OWNER = 8u
+  LOSSY_REPLICA_SKIP_OWNER = 8u,
+  /* Packets shorter than a tile of the fused step: use the packed bulk-copy build (one bulk copy per worker and
+   * tile, dropped sub-packets fetched too) where the launch policy allows it, instead of the gather pipeline
+   * (per-lane asynchronous copies of the delivered sub-packets only). Same results; for comparison and tests. */
+  LOSSY_PACKED_BULK = 16u
 };
 
 #define LOSSY_MAX_WORKERS 64u

@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "liblossy_b200.so")
 SOURCES = ["lossy_api.cu", "lossy_noalloc.cu"]
-HEADERS = ["lossy_device.cuh", "lossy_kernels.cuh", "lossy_tma.cuh", "lossy_phase_tma.cuh", os.path.join("..", "..", "include", "lossy.h")]
+HEADERS = ["lossy_device.cuh", "lossy_kernels.cuh", "lossy_tma.cuh", "lossy_gather.cuh", "lossy_phase_tma.cuh", os.path.join("..", "..", "include", "lossy.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -9,6 +9,7 @@
 #include <mutex>
 #include <new>
 
+#include "lossy_gather.cuh"
 #include "lossy_phase_tma.cuh"
 
 using namespace lossy;
@@ -279,12 +280,122 @@ int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
                : dispatch_tma<false, CW, GS, 0, PACKED, SPLIT>(ctx, P, G, s, blocks);
 }
 
+// ---- gather pipeline (packets shorter than a tile) ------------------------------------------
+// barriers, the ring of tile masks, stage headers; the drift sums per compute warp, the wire ring and the stages follow
+constexpr uint32_t kGatherSmemFixed = kGatherBarBytes + kGatherRing * sizeof(TileMasks) + kGatherMaxStages * sizeof(StageHdr);
+
+// few workers (twin geometry): the replica warps read the stale copies for the drift norms
+template <int CW>
+bool gather_rd(const lossy_config& c) { return CW == 8 && c.W <= kRdMaxWorkers; }
+
+template <int CW>
+bool gather_geometry(const lossy_ctx* ctx, bool drift, TmaGeom& G) {
+  constexpr uint32_t kTile = GatherShape<CW>::kTile;
+  const lossy_config& c = ctx->cfg;
+  const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
+  if (kfull == 0 || kfull >= (1ull << 31)) return false;
+  // whole packets per tile: powers of two from 128 elements that divide the tile, at most kMaxSub of them
+  const uint32_t P = c.packet_elems;
+  if (P >= kTile || (P & (P - 1u)) != 0 || P < 128u || kTile / P > (uint32_t)kMaxSub) return false;
+  memset(&G, 0, sizeof G);
+  G.packets_per_tile = kTile / P;
+  G.full_packets = (uint32_t)kfull;
+  const uint32_t gb = c.grad_dtype == LOSSY_BF16 ? 2 : 4, rb = c.replica_dtype == LOSSY_BF16 ? 2 : 4;
+  G.grad_slots = c.W < 8u ? c.W : 8u;
+  G.groups = (c.W + 7u) / 8u;
+  // a stage holds the group's gradient rows and theta, m, v
+  G.stage_bytes = (G.grad_slots * kTile * gb + 3 * kTile * 4 + 127u) & ~127u;
+  // fp64 drift sums per compute warp and replica, the wire ring, and (few workers, drift norms) the replica warps' scratch
+  G.state_bytes = CW * kMaxW * (uint32_t)sizeof(double) + kWireRing * kTile * rb;
+  if (drift && gather_rd<CW>(c)) G.state_bytes += GatherShape<CW>::kReplicaWarps * 2u * rd_buffer_bytes<CW>(rb);
+  const uint32_t budget = (227u * 1024u) / GatherShape<CW>::kCtasPerSm - 1024u;
+  const uint32_t avail = (uint32_t)ctx->smem_optin < budget ? (uint32_t)ctx->smem_optin : budget;
+  if (avail < kGatherSmemFixed + G.state_bytes + 2 * G.stage_bytes) return false;
+  G.stages = (avail - kGatherSmemFixed - G.state_bytes) / G.stage_bytes;
+  if (G.stages > 4u) G.stages = 4u;                           // more measured no faster (W = 2..32)
+  G.tiles_per_packet = 1;
+  const uint64_t tiles = (kfull + G.packets_per_tile - 1) / G.packets_per_tile;
+  if (tiles >= (1ull << 31)) return false;
+  G.num_tiles = (uint32_t)tiles;
+  G.status = ctx->status;
+  G.hints = 0;
+  return true;
+}
+
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, bool RD>
+int launch_gather(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks_out) {
+  auto kern = lossy_fused_gather_kernel<GT, RT, OPT, DRIFTK, CW, RD>;
+  const uint32_t smem = kGatherSmemFixed + G.state_bytes + G.stages * G.stage_bytes;
+  uint32_t blocks = (uint32_t)(ctx->num_sms * GatherShape<CW>::kCtasPerSm);
+  if (blocks > G.num_tiles) blocks = G.num_tiles;
+  *blocks_out = blocks;
+  if (ctx->plan_only) return LOSSY_OK;
+  static bool opted_in[kMaxDevices];   // per kernel instantiation and device: raise the dynamic shared memory limit once
+  cudaError_t e;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mu);
+    if (ctx->device >= kMaxDevices || !opted_in[ctx->device]) {
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tma_smem_budget<CW>(ctx));
+      if (e != cudaSuccess) return fail_cuda(ctx, "shared memory opt-in", e);
+      if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
+    }
+  }
+  kern<<<blocks, GatherShape<CW>::kThreads, smem, s>>>(P, G);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail_cuda(ctx, "gather kernel launch", e);
+  ctx->launches++;
+  return LOSSY_OK;
+}
+
+template <bool DRIFTK, int CW, bool RD>
+int dispatch_gather(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_t s, uint32_t* blocks) {
+  const bool gb = ctx->cfg.grad_dtype == LOSSY_BF16;
+  const bool rb = ctx->cfg.replica_dtype == LOSSY_BF16;
+  const bool adam = ctx->cfg.optimizer == LOSSY_ADAM;
+  if (gb && rb) return adam ? launch_gather<BF16, BF16, 1, DRIFTK, CW, RD>(ctx, P, G, s, blocks) : launch_gather<BF16, BF16, 0, DRIFTK, CW, RD>(ctx, P, G, s, blocks);
+  if (gb && !rb) return adam ? launch_gather<BF16, F32, 1, DRIFTK, CW, RD>(ctx, P, G, s, blocks) : launch_gather<BF16, F32, 0, DRIFTK, CW, RD>(ctx, P, G, s, blocks);
+  if (!gb && rb) return adam ? launch_gather<F32, BF16, 1, DRIFTK, CW, RD>(ctx, P, G, s, blocks) : launch_gather<F32, BF16, 0, DRIFTK, CW, RD>(ctx, P, G, s, blocks);
+  return adam ? launch_gather<F32, F32, 1, DRIFTK, CW, RD>(ctx, P, G, s, blocks) : launch_gather<F32, F32, 0, DRIFTK, CW, RD>(ctx, P, G, s, blocks);
+}
+
+template <int CW>
+int try_gather(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
+  TmaGeom G = {};
+  if (!gather_geometry<CW>(ctx, drift, G)) return LOSSY_OK;
+  *used = true;
+  if (ctx->plan)
+    snprintf(ctx->plan, ctx->plan_size, "gather %s packets/tile=%u stages=%u", CW == 16 ? "wide" : "twin", G.packets_per_tile, G.stages);
+  if constexpr (CW == 8) {
+    if (drift && gather_rd<CW>(ctx->cfg)) return dispatch_gather<true, CW, true>(ctx, P, G, s, blocks);
+  }
+  return drift ? dispatch_gather<true, CW, false>(ctx, P, G, s, blocks) : dispatch_gather<false, CW, false>(ctx, P, G, s, blocks);
+}
+
 // Run the build the policy picks; *used stays false when no bulk-copy launch fits (packets shorter
 // than a tile, or no complete packet): the register path then takes everything.
 int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
   *used = false;
   if (ctx->cfg.flags & LOSSY_REGISTER_PATH) return LOSSY_OK;
   const TmaPolicy t = tma_policy(ctx->cfg);
+  if (!(ctx->cfg.flags & LOSSY_PACKED_BULK) && ctx->cfg.packet_elems < (uint32_t)TmaShape<8>::kTile) {
+    // Packets shorter than a tile (128, 256 or 512 elements): the gather pipeline, where it beats the register
+    // kernel (fractions of the copy rate at 256 elements, W = 6..64): up to eight workers at every loss rate
+    // (0.72-0.98 against 0.60-0.92 for the packed bulk-copy build); more workers up to moderate loss
+    // (p = 0.05: 0.91-0.98 against 0.89-0.93); at high loss with many workers the register kernel stays ahead
+    // (p = 0.3, W >= 12: 0.71-0.77 against 0.65-0.77; p = 0.2, W = 32: 0.85 against 0.79). Few workers (W <= 4)
+    // run the twin geometry, whose replica warps also read the stale copies; the rest the wide one, where a
+    // packet allows it (256 elements and up).
+    const lossy_config& c = ctx->cfg;
+    const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
+    const bool reg_ahead = (c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15);
+    if (!reg_ahead) {
+      int rc = LOSSY_OK;
+      if (c.W > kRdMaxWorkers) rc = try_gather<16>(ctx, P, drift, s, blocks, used);
+      if (rc || *used) return rc;
+      rc = try_gather<8>(ctx, P, drift, s, blocks, used);
+      if (rc || *used) return rc;
+    }
+  }
   {
     // Packets of exactly half a wide tile with 13..16 workers at low loss: the PACKED wide build (two packets
     // per tile, one CTA per SM) beats the twin build, whose pieces are 2 KB (W = 16: 0.96-0.98 against 0.93 up
@@ -524,7 +635,7 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   if (cfg->packet_elems == 0 || cfg->packet_elems % 8 != 0) return LOSSY_EINVAL;
   if (!(cfg->p_grad >= 0.0 && cfg->p_grad < 1.0) || !(cfg->p_param >= 0.0 && cfg->p_param < 1.0)) return LOSSY_EINVAL;
   if (cfg->grad_dtype > LOSSY_BF16 || cfg->replica_dtype > LOSSY_BF16 || cfg->optimizer > LOSSY_ADAM) return LOSSY_EINVAL;
-  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH | LOSSY_REPLICA_SKIP_OWNER))
+  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH | LOSSY_REPLICA_SKIP_OWNER | LOSSY_PACKED_BULK))
     return LOSSY_EINVAL;
   const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
   const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;

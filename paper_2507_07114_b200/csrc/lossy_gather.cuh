@@ -1,0 +1,600 @@
+// Fused lossy step for packets SHORTER than a tile: the "gather" pipeline (sm_100a).
+//
+// A tile holds 2, 4 or 8 whole packets ("sub-packets"), each with delivery masks of its own, so every stream
+// of the step has holes at sub-packet granularity: dropped gradient pieces are not read, replicas that miss
+// a broadcast are not written, and their old copies are read for the drift term. Bulk copies of a few
+// hundred bytes are bound by their issue rate, not by memory, and a worker's whole tile piece in one bulk
+// copy reads the dropped sub-packets too. Here everything with holes moves as 16 bytes per lane (512 bytes per
+// warp instruction, whole lines), each lane testing the sub-packet its bytes lie in; only theta / m / v, which
+// have no holes, stay bulk copies. Roles of a CTA:
+//   mask warp      evaluates the delivery draws of a tile's sub-packets several tiles ahead and publishes them
+//                  in a ring of kGatherRing entries (also the optional count / bit-set outputs)
+//   gather warps   per tile and group of up to eight workers: asynchronous copies (cp.async, global -> shared
+//                  memory without passing through registers) of the DELIVERED pieces, completing on the stage's
+//                  mbarrier (cp.async.mbarrier.arrive.noinc); theta / m / v ride along as bulk copies
+//   compute warps  sum the pieces in ascending worker order, divide by the received count, run the optimizer
+//                  in place in shared memory, and write the wire tile into a ring of its own
+//   store warp     theta / m / v back with three bulk copies; releases the stage
+//   replica warps  each owns a fixed share of the replicas: from the wire ring it stores every (replica,
+//                  sub-packet) pair that takes the broadcast, and (drift norms) loads the old copy of every pair
+//                  that misses it and accumulates the squared difference — decoupled from the tile pipeline, so
+//                  no compute warp ever waits on a global load
+// A compute warp's 128 elements lie inside one sub-packet (packets here are powers of two from 128 elements
+// that divide the tile). Every wait is bounded as in the other pipelines. No cluster, no multicast.
+#pragma once
+#include "lossy_tma.cuh"
+
+namespace lossy {
+
+constexpr uint32_t kGatherRing = 8;     // tiles whose masks may be published ahead of the replica warps
+constexpr uint32_t kWireRing = 4;       // wire tiles between the compute warps and the replica warps
+template <int CW> struct GatherShape {
+  static constexpr int kProducers = CW >= 16 ? 2 : 1;                     // gather warps
+  static constexpr int kReplicaWarps = CW >= 16 ? 4 : 2;
+  static constexpr int kThreads = (CW + 2 + kProducers + kReplicaWarps) * 32;   // compute + mask + gather + store + replica
+  static constexpr int kTile = CW * 32 * kEpl;
+  static constexpr int kCtasPerSm = CW >= 16 ? 1 : 2;
+};
+constexpr uint32_t kRdMaxWorkers = 4;   // RD builds (below) serve at most this many workers
+// RD builds: bytes of one scratch buffer of a replica warp = the rows of all the replicas it can own
+template <int CW> __host__ __device__ constexpr uint32_t rd_buffer_bytes(uint32_t replica_elem_bytes) {
+  return ((kRdMaxWorkers + GatherShape<CW>::kReplicaWarps - 1u) / GatherShape<CW>::kReplicaWarps) *
+         (uint32_t)GatherShape<CW>::kTile * replica_elem_bytes;
+}
+constexpr uint32_t kGatherMaxStages = 8;    // a tile of few workers is small: more of them in flight
+constexpr uint32_t kGatherBarBytes = 512;   // 3 barriers per stage, 2 per mask-ring and wire-ring entry (8 B each), the abort flag
+static_assert((3 * kGatherMaxStages + 2 * kGatherRing + 2 * kWireRing) * 8 + 4 <= kGatherBarBytes, "barrier area too small");
+
+struct __align__(16) TileMasks {        // one ring entry: what the mask warp publishes about a tile
+  uint64_t recv[kMaxSub];               // per sub-packet: bit i = worker i's piece was delivered
+  uint64_t stale[kMaxSub];              // per sub-packet: bit i = replica i misses the broadcast
+  uint32_t j[kMaxSub];                  // per sub-packet: owner
+  uint64_t e0;                          // first element of the tile
+  uint32_t npk, len;                    // sub-packets and elements of the tile
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// the executing thread's earlier cp.async copies, once complete, count as one arrival on the barrier
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// One lane's arithmetic at the end of a tile: estimate = sum / count (Algorithm 1 mode: the saved aggregate
+// on a drop), the optimizer in place in shared memory, the wire value written once into `wire_tile` and returned widened.
+template <class RT, int OPT>
+__device__ __forceinline__ void finish_tile_lane(const Params& P, float (&acc)[kEpl], uint32_t cnt, unsigned char* sb,
+                                                 uint32_t off_th, uint32_t off_m, uint32_t off_v, unsigned char* wire_tile,
+                                                 uint32_t idx, uint64_t e, float (&wire)[kEpl]) {
+  divide_by_count<kEpl>(acc, cnt);
+  if (P.ghat_prev) {
+    uint32_t pw[4];
+    if (cnt == 0) {
+      load_words_stream<kEpl>(P.ghat_prev + e, pw);
+      unpack_lane<F32>(pw, acc);
+    } else {
+#pragma unroll
+      for (int x = 0; x < kEpl; ++x) pw[x] = __float_as_uint(acc[x]);
+      __stcs(reinterpret_cast<uint4*>(P.ghat_prev + e), make_uint4(pw[0], pw[1], pw[2], pw[3]));
+    }
+  }
+  if (P.ghat) {
+    uint32_t gw[4];
+#pragma unroll
+    for (int x = 0; x < kEpl; ++x) gw[x] = __float_as_uint(acc[x]);
+    store_words<kEpl>(P.ghat + e, gw);
+  }
+  float th[kEpl], m[kEpl], v[kEpl];
+  lds_lane<F32>(sb + off_th, idx, th);
+  if (!((P.flags & kZeroSkip) && cnt == 0)) {
+    if constexpr (OPT == 1) {
+      lds_lane<F32>(sb + off_m, idx, m);
+      lds_lane<F32>(sb + off_v, idx, v);
+    }
+    optimizer_n<OPT, kEpl>(P, acc, th, m, v);
+    sts_lane_f32(sb + off_th, idx, th);
+    if constexpr (OPT == 1) {
+      sts_lane_f32(sb + off_m, idx, m);
+      sts_lane_f32(sb + off_v, idx, v);
+    }
+  }
+  if constexpr (RT::kVecs == 2) {
+    sts_lane_f32(wire_tile, idx, th);
+#pragma unroll
+    for (int x = 0; x < kEpl; ++x) wire[x] = th[x];
+  } else {
+    uint32_t ww[4];
+    pack_bf16_lane(th, ww);
+    store_words<kEpl / 2>(wire_tile + (size_t)idx * 2, ww);
+    unpack_lane<BF16>(ww, wire);
+  }
+}
+
+// RD (drift norms with few replicas): the replica warps, not the compute warps, read the old copies of the
+// stale (replica, sub-packet) pairs — with asynchronous copies into a double-buffered scratch, requested one
+// tile ahead. With few workers the compute warps are bound by their issue slots and a tile is short, so that
+// neither their instruction budget nor the tile's duration hides those loads; with many replicas the scratch
+// would not fit and the sixteen compute warps' early requests hide them better.
+template <class GT, class RT, int OPT, bool DRIFTK, int CW, bool RD = false>
+__global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kCtasPerSm)
+    lossy_fused_gather_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
+  static_assert(!RD || DRIFTK, "RD is a way of computing the drift norms");
+  constexpr bool kWarpDrift = DRIFTK && !RD;               // the compute warps read the stale copies
+  constexpr int kTile = GatherShape<CW>::kTile;
+  constexpr int kNP = GatherShape<CW>::kProducers;
+  constexpr int kNR = GatherShape<CW>::kReplicaWarps;
+  constexpr int kGroup = 8;
+  constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
+  constexpr uint32_t kRowG = kTile * kGB, kRowR = kTile * kRB;          // bytes of one worker's / replica's row of a tile
+  extern __shared__ __align__(128) unsigned char smem[];
+  // layout: barriers | abort flag (kGatherBarBytes) | ring of tile masks | stage headers | fp64 drift sums per compute
+  //         warp and replica | wire ring | stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kGatherBarBytes - 4);
+  TileMasks* ring = reinterpret_cast<TileMasks*>(smem + kGatherBarBytes);
+  StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + kGatherBarBytes + kGatherRing * sizeof(TileMasks));
+  double* warp_acc = reinterpret_cast<double*>(smem + kGatherBarBytes + kGatherRing * sizeof(TileMasks) + kGatherMaxStages * sizeof(StageHdr));
+  unsigned char* wring = reinterpret_cast<unsigned char*>(warp_acc + CW * kMaxW);
+  constexpr uint32_t kRdBuf = rd_buffer_bytes<CW>(kRB);
+  unsigned char* rscratch = wring + kWireRing * kRowR;     // RD: two buffers per replica warp
+  unsigned char* stage0 = rscratch + (RD ? kNR * 2u * kRdBuf : 0u);
+  const uint32_t S = G.stages;
+  const uint32_t off_th = G.grad_slots * kRowG;
+  const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4;
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const uint32_t W = P.W;
+  const uint32_t lgP = 31u - (uint32_t)__clz((int)P.P);                 // packets are powers of two here
+  auto full_bar = [&](uint32_t s) { return smem_u32(&bars[s]); };
+  auto done_bar = [&](uint32_t s) { return smem_u32(&bars[kGatherMaxStages + s]); };
+  auto empty_bar = [&](uint32_t s) { return smem_u32(&bars[2 * kGatherMaxStages + s]); };
+  auto mfull_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kGatherMaxStages + q]); };
+  auto mempty_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kGatherMaxStages + kGatherRing + q]); };
+  auto wfull_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kGatherMaxStages + 2 * kGatherRing + q]); };
+  auto wempty_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kGatherMaxStages + 2 * kGatherRing + kWireRing + q]); };
+
+  for (uint32_t q = threadIdx.x; q < (uint32_t)CW * kMaxW; q += blockDim.x) warp_acc[q] = 0.0;
+  if (threadIdx.x == 0) {
+    *abort_flag = 0u;
+    for (uint32_t s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 32u * kNP + 1u);        // every gather lane's copies, and the header's writer
+      mbar_init(done_bar(s), CW);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (uint32_t q = 0; q < kGatherRing; ++q) {
+      mbar_init(mfull_bar(q), 1);
+      mbar_init(mempty_bar(q), kNR);                 // the replica warps are the last readers of a tile's masks
+    }
+    for (uint32_t q = 0; q < kWireRing; ++q) {
+      mbar_init(wfull_bar(q), CW);
+      mbar_init(wempty_bar(q), kNR);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  __syncthreads();
+
+  if (warp == CW) {
+    // ================================= mask warp =================================
+    uint32_t slot = 0, par = 0;
+    uint32_t Wp = 32;
+    const bool batched = W <= 32 && !P.ghat_prev;          // Algorithm 1 draws once per packet
+    if (batched) { Wp = 1; while (Wp < W) Wp <<= 1; }
+    const uint32_t lgWp = 31u - (uint32_t)__clz((int)Wp);
+    const uint32_t Bp = 32u >> lgWp;                        // sub-packets per pass of draws
+    const uint32_t wmask = Wp == 32 ? 0xFFFFFFFFu : ((1u << Wp) - 1u);
+    // the old copy of a (replica, sub-packet) pair that misses the broadcast is read by a compute warp several
+    // tiles later for the drift term: start it toward L2 now (one bulk prefetch per pair)
+    auto prefetch_stale = [&](uint32_t i, uint32_t j, uint32_t k) {
+      bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, j, (uint64_t)k * P.P), P.P * kRB);
+    };
+    for (uint32_t tile = blockIdx.x; tile < G.num_tiles; tile += gridDim.x) {
+      if (!mbar_wait(mempty_bar(slot), par ^ 1u, abort_flag)) break;
+      const uint32_t kfirst = tile * G.packets_per_tile;
+      const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
+      TileMasks& tm = ring[slot];
+      auto report = [&](uint32_t sp, uint32_t j, uint64_t r, uint64_t st, uint64_t gbad, uint64_t pbad) {   // one lane
+        const uint32_t k = kfirst + sp;
+        tm.recv[sp] = r;
+        tm.stale[sp] = st;
+        tm.j[sp] = j;
+        if (P.count) P.count[k] = (uint8_t)__popcll(r);
+        if (P.recv_bits) P.recv_bits[k] = r;
+        if (P.stale_bits) P.stale_bits[k] = st;
+        if (P.burst_out) {
+          P.burst_out[k] = gbad;
+          P.burst_out[(size_t)P.K + k] = pbad;
+        }
+      };
+      if (batched) {
+        for (uint32_t q0 = 0; q0 < npk; q0 += Bp) {
+          const uint32_t sp_l = q0 + ((uint32_t)lane >> lgWp), i_l = (uint32_t)lane & (Wp - 1u);
+          const uint32_t k_l = kfirst + (sp_l < npk ? sp_l : 0u);
+          const uint32_t j_l = (P.k0 + k_l) / P.pps;
+          const BatchDraws d = batch_draws<AGG | BCAST>(P, k_l, j_l, i_l, sp_l < npk && i_l < W);
+          uint64_t st_l = 0;                                 // the stale set of this lane's own sub-packet
+          for (uint32_t x = 0; x < Bp && q0 + x < npk; ++x) {
+            uint64_t r, st, gbad, pbad;
+            batch_masks<AGG | BCAST>(P, d, kfirst + q0 + x, (int)(x * Wp), wmask, r, st, gbad, pbad);
+            const uint32_t j_x = __shfl_sync(0xFFFFFFFFu, j_l, (int)(x * Wp));
+            if (x == ((uint32_t)lane >> lgWp)) st_l = st;
+            if ((uint32_t)lane == x) report(q0 + x, j_x, r, st, gbad, pbad);
+          }
+          if constexpr (kWarpDrift) {
+            if (sp_l < npk && i_l < W && ((st_l >> i_l) & 1ull)) prefetch_stale(i_l, j_l, k_l);
+          }
+        }
+      } else {
+        for (uint32_t sp = 0; sp < npk; ++sp) {
+          uint64_t r, st, gbad, pbad;
+          const uint32_t j_sp = (P.k0 + kfirst + sp) / P.pps;
+          packet_masks<AGG | BCAST>(P, kfirst + sp, j_sp, lane, r, st, gbad, pbad);
+          if (lane == 0) report(sp, j_sp, r, st, gbad, pbad);
+          if constexpr (kWarpDrift) {
+            for (uint32_t i = lane; i < W; i += 32)
+              if ((st >> i) & 1ull) prefetch_stale(i, j_sp, kfirst + sp);
+          }
+        }
+      }
+      if ((uint32_t)lane >= npk && lane < kMaxSub) {      // entries behind a short last tile: nothing delivered, nothing to do
+        tm.recv[lane] = 0;
+        tm.stale[lane] = ~0ull;
+        tm.j[lane] = 0;
+      }
+      if (lane == 0) {
+        tm.e0 = (uint64_t)kfirst * P.P;
+        tm.npk = npk;
+        tm.len = npk * P.P;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(mfull_bar(slot));
+      if (++slot == kGatherRing) { slot = 0; par ^= 1u; }
+    }
+  } else if (warp > CW && warp <= CW + kNP) {
+    // ================================ gather warps ================================
+    const uint32_t pw = (uint32_t)(warp - CW - 1);          // which gather warp
+    uint32_t s = 0, par = 0, slot = 0, mpar = 0;
+    bool ok = true;
+    auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      if (!mbar_wait(mfull_bar(slot), mpar, abort_flag)) { ok = false; break; }
+      const TileMasks& tm = ring[slot];
+      const uint64_t e0 = tm.e0;
+      const uint32_t len = tm.len;
+      // lane l holds sub-packet (l & 7)'s receive mask; a ballot per worker turns that column into the worker's
+      // row of delivered sub-packets
+      const uint64_t recv_l = tm.recv[lane & (kMaxSub - 1)];
+      for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
+        if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
+        const bool last = g + 1 == G.groups;
+        const uint32_t in_group = min((uint32_t)kGroup, W - g * kGroup);
+        const uint32_t st = smem_u32(stage0 + (size_t)s * G.stage_bytes);
+        if (pw == 0) {
+          // the header, and theta / m / v as three bulk copies on the same barrier
+          if (lane == 0) {
+            StageHdr& h = hdrs[s];
+            h.recv = 0; h.stale = 0; h.e0 = e0; h.k = slot; h.len = len; h.cnt = 0; h.last = last ? 1u : 0u; h.own = 0; h.j = 0;
+            if (last) mbar_arrive_expect_tx(full_bar(s), (OPT == 1 ? 3u : 1u) * len * 4u);   // publishes the header
+            else mbar_arrive(full_bar(s));
+          }
+          __syncwarp();
+          if (last) {
+            if (lane == 8) bulk_g2s(st + off_th, P.master + e0, len * 4u, full_bar(s), false, 0);
+            if constexpr (OPT == 1) {
+              if (lane == 9) bulk_g2s(st + off_m, P.m + e0, len * 4u, full_bar(s), false, 0);
+              if (lane == 10) bulk_g2s(st + off_v, P.v + e0, len * 4u, full_bar(s), false, 0);
+            }
+          }
+        }
+        // Delivered pieces of this group's workers: a row is copied in chunks of 512 bytes (one warp
+        // instruction, 16 bytes per lane), each lane testing the sub-packet its 16 bytes lie in.
+        for (uint32_t u = 0; u < in_group; ++u) {
+          const uint32_t rowmask = __ballot_sync(0xFFFFFFFFu, (recv_l >> (g * kGroup + u)) & 1ull) & 0xFFu;
+          if (rowmask == 0u) continue;
+          const unsigned char* src = reinterpret_cast<const unsigned char*>(P.grads[g * kGroup + u]) + e0 * kGB;
+          const uint32_t dst = st + u * kRowG;
+#pragma unroll
+          for (uint32_t c = pw; c < kRowG / 512u; c += kNP) {
+            const uint32_t off = c * 512u + (uint32_t)lane * 16u;   // byte within the row
+            if ((rowmask >> ((off / kGB) >> lgP)) & 1u) cp_async16(dst + off, src + off);
+          }
+        }
+        cp_async_arrive(full_bar(s));
+      }
+      if (++slot == kGatherRing) { slot = 0; mpar ^= 1u; }
+    }
+    // copies in flight at an abort: wait for this warp's own before the CTA exits
+    if (!ok || *abort_flag) asm volatile("cp.async.wait_all;" ::: "memory");
+  } else if (warp == CW + kNP + 1) {
+    // ================================ store warp =================================
+    uint32_t s = 0, par = 0;
+    bool ok = true;
+    const bool sh_hint = G.hints & 2u;
+    const uint64_t pol = policy_evict_first();
+    auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
+        if (!mbar_wait(done_bar(s), par, abort_flag)) { ok = false; break; }
+        if (g + 1 == G.groups) {
+          const uint64_t e0 = hdrs[s].e0;
+          const uint32_t len = hdrs[s].len;
+          unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+          if (lane == 0) bulk_s2g(P.master + e0, smem_u32(st + off_th), len * 4u, sh_hint, pol);
+          if constexpr (OPT == 1) {
+            if (lane == 1) bulk_s2g(P.m + e0, smem_u32(st + off_m), len * 4u, sh_hint, pol);
+            if (lane == 2) bulk_s2g(P.v + e0, smem_u32(st + off_v), len * 4u, sh_hint, pol);
+          }
+          bulk_commit();
+          bulk_wait_read0();          // shared memory of this stage may be overwritten after this
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar(s));
+      }
+    }
+    bulk_wait0();
+  } else if (warp > CW + kNP + 1) {
+    // =============================== replica warps ===============================
+    const uint32_t rw = (uint32_t)(warp - CW - kNP - 2);    // this warp owns replicas rw, rw + kNR, ...
+    constexpr int kChunks = kRowR / 512u;                   // a replica's row of a tile in 512-byte chunks
+    constexpr uint32_t kElemsPerChunk = 512u / kRB;
+    unsigned char* scratch = rscratch + (size_t)rw * 2u * kRdBuf;
+    uint32_t slot = 0, wslot = 0, wpar = 0, mpar = 0, buf = 0;
+    // RD: PASS 0 requests the old copies of a tile's stale (replica, sub-packet) pairs into scratch buffer `b`
+    // (chunk after chunk in the order (replica, chunk)); pass 1 takes their squared differences against the wire
+    // tile: fp32 per lane within a replica's chunks, one warp reduction per replica and tile, fp64 from there on
+    // (each replica has one accumulator, touched by this warp alone, in tile order).
+    auto drift_pass = [&](const TileMasks& tm, uint32_t b, int pass, const unsigned char* wt) {
+      const uint64_t stale_l = tm.stale[lane & (kMaxSub - 1)];
+      const uint32_t j_l = tm.j[lane & (kMaxSub - 1)];
+      const uint32_t live_tile = (1u << tm.npk) - 1u;       // entries behind a short last tile are marked stale everywhere
+      const uint64_t e0 = tm.e0;
+      uint32_t n = 0;                                       // chunks with a stale sub-packet met so far (warp-uniform)
+      for (uint32_t i = rw; i < W; i += kNR) {
+        const uint32_t live = __ballot_sync(0xFFFFFFFFu, (stale_l >> i) & 1ull) & 0xFFu & live_tile;
+        if (live == 0u) continue;
+        const unsigned char* base = reinterpret_cast<const unsigned char*>(P.replicas[i]);
+        float sq = 0.0f;
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const uint32_t el0 = (uint32_t)c * kElemsPerChunk;                    // the chunk's sub-packets, as bits
+          const uint32_t in_chunk = ((2u << ((el0 + kElemsPerChunk - 1u) >> lgP)) - 1u) & ~((1u << (el0 >> lgP)) - 1u);
+          if ((live & in_chunk) == 0u) continue;
+          const uint32_t q = n++;
+          const uint32_t off = (uint32_t)c * 512u + (uint32_t)lane * 16u;
+          const uint32_t el = off / kRB, sp = el >> lgP;
+          const uint32_t j_sp = __shfl_sync(0xFFFFFFFFu, j_l, (int)sp);
+          const bool mine = (live >> sp) & 1u;                                  // this lane's 16 bytes are stale ones
+          unsigned char* sc = scratch + (size_t)b * kRdBuf + q * 512u + (uint32_t)lane * 16u;
+          if (pass == 0) {
+            if (mine) cp_async16(smem_u32(sc), base + rep_index(P, i, j_sp, e0 + el) * kRB);
+          } else if (mine) {
+            const uint4 ov = *reinterpret_cast<const uint4*>(sc);               // each lane reads back what it copied itself
+            const uint4 wv = *reinterpret_cast<const uint4*>(wt + off);
+            const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w}, ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              if constexpr (RT::kVecs == 2) {              // fp32 replicas: one element per word
+                const float d0 = __fsub_rn(__uint_as_float(ow[h]), __uint_as_float(ww[h]));
+                sq = __fadd_rn(sq, __fmul_rn(d0, d0));
+              } else {                                      // bf16 replicas: two elements per word
+                const float d0 = __fsub_rn(__uint_as_float(ow[h] << 16), __uint_as_float(ww[h] << 16));
+                const float d1 = __fsub_rn(__uint_as_float(ow[h] & 0xFFFF0000u), __uint_as_float(ww[h] & 0xFFFF0000u));
+                sq = __fadd_rn(sq, __fmul_rn(d0, d0));
+                sq = __fadd_rn(sq, __fmul_rn(d1, d1));
+              }
+            }
+          }
+        }
+        if (pass == 1) {
+          const float tot = warp_sum(sq);
+          if (lane == 0) warp_acc[i] += (double)tot;        // row 0 of the sums: one accumulator per replica
+        }
+      }
+    };
+    if constexpr (RD) {
+      if (blockIdx.x < G.num_tiles) {
+        if (mbar_wait(mfull_bar(0), 0u, abort_flag)) drift_pass(ring[0], 0u, 0, nullptr);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    for (uint32_t tile = blockIdx.x; tile < G.num_tiles; tile += gridDim.x) {
+      if constexpr (RD) {
+        // the next tile's old copies first: they have this tile's duration to arrive
+        if (tile + gridDim.x < G.num_tiles) {
+          const uint32_t nslot = slot + 1u == kGatherRing ? 0u : slot + 1u;
+          if (!mbar_wait(mfull_bar(nslot), nslot == 0u ? mpar ^ 1u : mpar, abort_flag)) break;
+          drift_pass(ring[nslot], buf ^ 1u, 0, nullptr);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
+      // the wire tile is complete: every compute warp has arrived, and each had waited for the tile's masks first
+      if (!mbar_wait(wfull_bar(wslot), wpar, abort_flag)) break;
+      const TileMasks& tm = ring[slot];
+      const uint64_t e0 = tm.e0;
+      const unsigned char* wt = wring + (size_t)wslot * kRowR;
+      // lane l holds sub-packet (l & 7)'s masks; a ballot per replica turns that column into the replica's row
+      const uint32_t j_l = tm.j[lane & (kMaxSub - 1)];
+      const uint64_t keep_l = tm.stale[lane & (kMaxSub - 1)] | own_bit(P, j_l);   // not written: missed the broadcast, or does not exist
+      uint32_t jc[kChunks];                                 // owner of the sub-packet this lane's bytes of chunk c lie in
+#pragma unroll
+      for (int c = 0; c < kChunks; ++c)
+        jc[c] = __shfl_sync(0xFFFFFFFFu, j_l, (int)((((uint32_t)c * 512u + (uint32_t)lane * 16u) / kRB) >> lgP));
+      for (uint32_t i = rw; i < W; i += kNR) {
+        const uint32_t fresh = __ballot_sync(0xFFFFFFFFu, !((keep_l >> i) & 1ull)) & 0xFFu;   // bit sp: replica i takes it
+        if (fresh == 0u) continue;
+        unsigned char* base = reinterpret_cast<unsigned char*>(P.replicas[i]);
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const uint32_t off = (uint32_t)c * 512u + (uint32_t)lane * 16u;
+          const uint32_t el = off / kRB;
+          if ((fresh >> (el >> lgP)) & 1u)
+            __stcs(reinterpret_cast<uint4*>(base + rep_index(P, i, jc[c], e0 + el) * kRB),
+                   *reinterpret_cast<const uint4*>(wt + off));
+        }
+      }
+      if constexpr (RD) {
+        asm volatile("cp.async.wait_group 1;" ::: "memory");   // everything but the next tile's requests has landed
+        drift_pass(tm, buf, 1, wt);
+        buf ^= 1u;
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(wempty_bar(wslot));
+        mbar_arrive(mempty_bar(slot));
+      }
+      if (++slot == kGatherRing) { slot = 0; mpar ^= 1u; }
+      if (++wslot == kWireRing) { wslot = 0; wpar ^= 1u; }
+    }
+    if constexpr (RD) asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
+    // =============================== compute warps ===============================
+    const uint32_t idx = threadIdx.x * kEpl;               // first element of this lane within the tile
+    const uint32_t my_sp = ((uint32_t)(threadIdx.x & ~31) * kEpl) >> lgP;   // this warp's sub-packet, always the same
+    uint32_t s = 0, par = 0, slot = 0, mpar = 0, wslot = 0, wpar = 0;
+    bool ok = true;
+    float acc[kEpl];
+    auto next_stage = [&]() { if (++s == S) { s = 0; par ^= 1u; } };
+    constexpr int kWords = LaneWords<RT>::value;
+    constexpr int kPre = 4;                                  // stale copies requested before the tile's arithmetic
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      if (!mbar_wait(mfull_bar(slot), mpar, abort_flag)) { ok = false; break; }
+      const TileMasks& tm = ring[slot];
+      const uint32_t len = tm.len;
+      const uint64_t e0 = tm.e0;
+      const bool active = idx < len;
+      const uint64_t my_recv = tm.recv[my_sp];             // zero behind a short last tile
+      // The old copies this warp compares against for the drift term (in L2 by now: the mask warp asked for them
+      // tiles ago) are requested first, so that their latency hides behind the wait for the tile and its arithmetic.
+      [[maybe_unused]] uint32_t pre_raw[kPre][4];
+      [[maybe_unused]] int pre_id[kPre];
+      [[maybe_unused]] uint32_t my_j = 0;
+      uint64_t stale_rest = 0;
+      if constexpr (kWarpDrift) {
+        if (active) {
+          stale_rest = tm.stale[my_sp];
+          my_j = tm.j[my_sp];
+        }
+#pragma unroll
+        for (int b = 0; b < kPre; ++b) {
+          pre_id[b] = -1;
+          if (stale_rest) {
+            pre_id[b] = __ffsll((long long)stale_rest) - 1;
+            stale_rest &= stale_rest - 1;
+            load_words_stream<kWords>(reinterpret_cast<const typename RT::raw*>(P.replicas[pre_id[b]]) +
+                                          rep_index(P, (uint32_t)pre_id[b], my_j, e0 + idx), pre_raw[b]);
+          }
+        }
+      }
+#pragma unroll
+      for (int x = 0; x < kEpl; ++x) acc[x] = 0.0f;
+      for (uint32_t g = 0; g < G.groups; ++g, next_stage()) {
+        if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
+        unsigned char* st = stage0 + (size_t)s * G.stage_bytes;
+        const uint32_t bits = (uint32_t)(my_recv >> (g * kGroup)) & 0xFFu;
+#pragma unroll
+        for (int u = 0; u < kGroup; ++u)
+          if ((bits >> u) & 1u) {
+            float f[kEpl];
+            lds_lane<GT>(st + (size_t)u * kRowG, idx, f);
+#pragma unroll
+            for (int x = 0; x < kEpl; ++x) acc[x] = __fadd_rn(acc[x], f[x]);
+          }
+        if (g + 1 == G.groups) {
+          // the wire tile goes into the ring the replica warps drain
+          if (!mbar_wait(wempty_bar(wslot), wpar ^ 1u, abort_flag)) { ok = false; break; }
+          float wire[kEpl];
+#pragma unroll
+          for (int x = 0; x < kEpl; ++x) wire[x] = 0.0f;
+          if (active)
+            finish_tile_lane<RT, OPT>(P, acc, (uint32_t)__popcll(my_recv), st, off_th, off_m, off_v,
+                                      wring + (size_t)wslot * kRowR, idx, e0 + idx, wire);
+          fence_proxy_async();          // make theta / m / v visible to the bulk stores
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(wfull_bar(wslot));
+            mbar_arrive(done_bar(s));
+          }
+          if (++wslot == kWireRing) { wslot = 0; wpar ^= 1u; }
+          if constexpr (kWarpDrift) {
+            // squared differences of up to four copies at a time, their warp totals in one multi-value reduction;
+            // the first lane of segment b adds copy b's total to this warp's fp64 sum of that replica
+            auto reduce4 = [&](float (&sq)[4], const int (&ids)[4]) {
+              const float tot = warp_sum_multi<4>(sq, lane);
+              const int b = lane >> 3;
+              int id = ids[0];
+#pragma unroll
+              for (int x = 1; x < 4; ++x) id = b == x ? ids[x] : id;
+              if ((lane & 7) == 0 && id >= 0) warp_acc[warp * kMaxW + id] += (double)tot;
+            };
+            if (pre_id[0] >= 0) {     // warp-uniform: the warp's elements lie in one sub-packet
+              float sq[4];
+#pragma unroll
+              for (int b = 0; b < kPre; ++b) {
+                sq[b] = 0.0f;
+                if (pre_id[b] >= 0) {
+                  float old[kEpl];
+                  unpack_lane<RT>(pre_raw[b], old);
+#pragma unroll
+                  for (int x = 0; x < kEpl; ++x) {
+                    const float d = __fsub_rn(old[x], wire[x]);
+                    sq[b] = __fadd_rn(sq[b], __fmul_rn(d, d));
+                  }
+                }
+              }
+              reduce4(sq, pre_id);
+              while (stale_rest) {     // more stale copies than were requested early
+                int ids[4];
+                uint32_t raw[4][4];
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                  ids[b] = -1;
+                  if (stale_rest) {
+                    ids[b] = __ffsll((long long)stale_rest) - 1;
+                    stale_rest &= stale_rest - 1;
+                    load_words_stream<kWords>(reinterpret_cast<const typename RT::raw*>(P.replicas[ids[b]]) +
+                                                  rep_index(P, (uint32_t)ids[b], my_j, e0 + idx), raw[b]);
+                  }
+                }
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                  sq[b] = 0.0f;
+                  if (ids[b] >= 0) {
+                    float old[kEpl];
+                    unpack_lane<RT>(raw[b], old);
+#pragma unroll
+                    for (int x = 0; x < kEpl; ++x) {
+                      const float d = __fsub_rn(old[x], wire[x]);
+                      sq[b] = __fadd_rn(sq[b], __fmul_rn(d, d));
+                    }
+                  }
+                }
+                reduce4(sq, ids);
+              }
+            }
+          }
+        } else {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(done_bar(s));
+        }
+      }
+      if (++slot == kGatherRing) { slot = 0; mpar ^= 1u; }
+    }
+  }
+
+  // ---- common exit: per-CTA drift partials in fixed order, status word ---------------
+  __syncthreads();
+  if (*abort_flag && threadIdx.x == 0) atomicExch(G.status, 1u);
+  if constexpr (DRIFTK) {
+    if (threadIdx.x < kMaxW) {
+      double t = 0.0;
+#pragma unroll
+      for (int w = 0; w < CW; ++w) t += warp_acc[w * kMaxW + threadIdx.x];
+      P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
+    }
+    if (P.ticket) drift_last_block(P, warp, lane, GatherShape<CW>::kThreads / 32);
+  }
+}
+
+}  // namespace lossy

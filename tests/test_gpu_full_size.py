@@ -118,11 +118,18 @@ def test_config5_point_full_size_small_packets_register_path():
     _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
 
 
-def test_config5_point_full_size_small_packets_packed_build():
-    # P=256 at low loss takes the PACKED bulk-copy build (eight whole packets per tile) at full size
-    w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.05)
-    gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
-    assert L.lossy_describe_plan(gpu.ctx).startswith("bulk-copy wide group=8 stale=late packed")
+def test_config5_point_full_size_small_packets_gather_pipeline():
+    # P=256 at low and moderate loss takes the gather pipeline (eight whole packets per tile) at full size
+    w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.1)
+    gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=True)
+    assert L.lossy_describe_plan(gpu.ctx) == "gather wide packets/tile=8 stages=3"
+
+
+def test_few_workers_small_packets_full_size_gather_twin():
+    # W = 4, P = 256 at high loss: the twin gather build whose replica warps also read the stale copies
+    w = workload.scaled(CFG["cfg2_w8_layer_adam"], workload.LAYER_ELEMS, W=4, packet_elems=256, p=0.3)
+    gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=True)
+    assert L.lossy_describe_plan(gpu.ctx) == "gather twin packets/tile=4 stages=4"
 
 
 def test_drift_is_order_one_and_matches_the_stationary_constant_at_scale():

@@ -1,6 +1,6 @@
 """Out-of-bounds check without a sanitizer: every buffer sits between two poisoned 4 KB bands that must
-come back untouched, on ragged sizes and on every kernel (bulk-copy wide / twin / packed, register path,
-unfused calls)."""
+come back untouched, on ragged sizes and on every kernel (bulk-copy wide / twin / packed, gather wide / twin,
+register path, unfused calls)."""
 import pytest
 import torch
 
@@ -35,8 +35,11 @@ CASES = [
     ("twin_w40_short_last_tile", 40, 1032 * 23 + 512, 1032, 0.2, "adam", "bf16", "f32", 0),
     ("twin_w64_split_staged", 64, 1024 * 30 + 16, 1024, 0.3, "adam", "bf16", "bf16", 0),
     ("packed_1024_two_per_wide_tile", 16, 1024 * 21 + 8, 1024, 0.05, "adam", "bf16", "bf16", 0),
-    ("packed_256", 16, 256 * 45 + 40, 256, 0.1, "adam", "bf16", "bf16", 0),
-    ("packed_128_twin", 30, 128 * 77 + 8, 128, 0.1, "sgd", "f32", "bf16", 0),
+    ("packed_256", 16, 256 * 45 + 40, 256, 0.1, "adam", "bf16", "bf16", L.LOSSY_PACKED_BULK),
+    ("packed_128_twin", 30, 128 * 77 + 8, 128, 0.1, "sgd", "f32", "bf16", L.LOSSY_PACKED_BULK),
+    ("gather_wide_256", 16, 256 * 45 + 40, 256, 0.1, "adam", "bf16", "bf16", 0),
+    ("gather_twin_128", 20, 128 * 77 + 8, 128, 0.1, "sgd", "f32", "bf16", 0),
+    ("gather_twin_few_workers_512", 3, 512 * 23 + 16, 512, 0.4, "adam", "bf16", "f32", 0),
     ("register_path", 8, 2048 * 7 + 5, 2048, 0.3, "adam", "bf16", "bf16", L.LOSSY_REGISTER_PATH),
     ("tiny_unaligned_tail", 3, 1029, 1000, 0.3, "sgd", "f32", "f32", 0),
 ]

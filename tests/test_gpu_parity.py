@@ -107,11 +107,16 @@ EDGE = [
 
 
 @pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
-@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("fused", [True, False, "packed_bulk"])
 def test_edge_cases(case, fused):
     name, W, n, P, p, opt, gd, rd, flags = case
+    if fused == "packed_bulk":
+        # small packets have two fused builds: the gather pipeline (default) and the packed bulk-copy build
+        if "packed" not in name:
+            pytest.skip("not a small-packet case")
+        flags |= L.LOSSY_PACKED_BULK
     w = workload.Workload(name, W, n, P, p, opt, 1e-2 if opt == "sgd" else 3e-4, gd, rd, 5, seed=42)
-    gpu, orc = run_parity(w, 5, fused=fused, flags=flags)
+    gpu, orc = run_parity(w, 5, fused=bool(fused), flags=flags)
     if name.startswith("heavy_loss") or name.startswith("bulk_zero"):
         assert int((gpu.count == 0).sum()) > 0          # the nothing-received fallback was exercised
 
@@ -191,7 +196,7 @@ def test_empty_bucket_is_a_noop_and_bad_arguments_are_rejected():
     assert L.lossy_kernel_launches(ctx) == 0
     L.lossy_destroy(ctx)
     for bad in (dict(W=0), dict(W=65), dict(packet_elems=0), dict(packet_elems=12), dict(p_grad=1.0),
-                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=16), dict(optimizer=5)):
+                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=32), dict(optimizer=5)):
         kw = dict(W=2, n=64, packet_elems=64, p_grad=0.1, p_param=0.1, seed=0, grad_dtype=torch.float32,
                   replica_dtype=torch.float32, optimizer="sgd", lr=0.1)
         kw.update(bad)
@@ -321,9 +326,13 @@ def test_launch_policy_picks_the_expected_build_for_the_benchmark_configurations
     assert plan(64, 4096, 0.1)[0] == "bulk-copy twin group=8 stale=late stages=3"         # config 3
     assert plan(4, 1024, 0.1, gd="f32", rd="f32")[0].startswith("bulk-copy twin group=4")  # config 1
     assert plan(16, 1024, 0.3)[0] == "bulk-copy twin group=8 stale=early stages=3"        # config 5, P = 1024
-    assert plan(16, 256, 0.1)[0].startswith("bulk-copy wide group=8 stale=late packed")   # config 5, small packets, low loss
+    assert plan(16, 256, 0.1)[0] == "gather wide packets/tile=8 stages=3"                  # config 5, small packets, low loss
     assert plan(16, 1024, 0.05)[0].startswith("bulk-copy wide group=8 stale=late packed")  # config 5, P = 1024, low loss: two packets per wide tile
-    assert plan(16, 256, 0.3)[0] == "register kernel"                                     # ... and at high loss
+    assert plan(16, 256, 0.3)[0] == "register kernel"                                     # ... and at high loss with many workers
+    assert plan(8, 256, 0.3)[0] == "gather wide packets/tile=8 stages=3"
+    assert plan(4, 256, 0.3)[0] == "gather twin packets/tile=4 stages=4"                  # few workers: twin geometry
+    assert plan(40, 128, 0.1)[0].startswith("gather twin packets/tile=8")                 # 128 elements: only the twin tile packs them
+    assert plan(16, 256, 0.1, flags=L.LOSSY_PACKED_BULK)[0].startswith("bulk-copy wide group=8 stale=late packed")
     assert plan(64, 4096, 0.3)[0] == "bulk-copy twin group=8 stale=staged split stages=4"
     assert plan(24, 2048, 0.2)[0] == "bulk-copy twin group=8 stale=early split stages=3"
     # fp32 replicas do not fit bf16 gradient slots: early requests instead of staged copies
@@ -341,7 +350,7 @@ def test_packed_build_many_tiles_per_cta_with_skewed_stale_sets():
     W, P = 8, 256
     n = 2048 * 148 * 40 + 256 * 3
     w = workload.Workload("packed_skew", W, n, P, 0.0, "adam", 3e-4, "bf16", "bf16", 4, seed=77)
-    gpu = GpuRun(w, p_grad=0.2, p_param=0.7)
+    gpu = GpuRun(w, flags=L.LOSSY_PACKED_BULK, p_grad=0.2, p_param=0.7)
     assert "packed" in L.lossy_describe_plan(gpu.ctx)
     orc = make_oracle(w, p_grad=0.2, p_param=0.7)
     K = w.K

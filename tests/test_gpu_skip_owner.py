@@ -12,6 +12,7 @@ from parity_util import GpuRun, REL_TOL, assert_rel, assert_same, make_oracle, r
 
 pytestmark = pytest.mark.gpu
 ELIDE, REG, SKIP, LOSSLESS = L.LOSSY_REPLICA_SKIP_OWNER, L.LOSSY_REGISTER_PATH, L.LOSSY_ZERO_SKIP, L.LOSSY_SELF_LOSSLESS
+PACKED = L.LOSSY_PACKED_BULK
 
 CASES = [
     # name, W, n, P, p, opt, gd, rd, extra flags, expected start of the plan (None = any)
@@ -20,10 +21,15 @@ CASES = [
     ("twin_w64", 64, 4096 * 70 + 40, 4096, 0.1, "adam", "bf16", "bf16", 0, "bulk-copy twin group=8 stale=late"),
     ("twin_split_staged_w64", 64, 1024 * 130 + 8, 1024, 0.3, "adam", "bf16", "bf16", 0, "bulk-copy twin group=8 stale=staged split"),
     ("twin_split_early_w24", 24, 1024 * 75, 1024, 0.2, "sgd", "f32", "f32", 0, "bulk-copy twin group=8 stale=early split"),
-    ("packed_wide_256", 16, 256 * 61 + 40, 256, 0.1, "adam", "bf16", "bf16", 0, "bulk-copy wide group=8 stale=late packed"),
-    ("packed_twin_128_w40", 40, 128 * 90 + 8, 128, 0.3, "sgd", "bf16", "bf16", 0, "bulk-copy twin group=8 stale=late packed"),
-    ("packed_512_w3_f32", 3, 512 * 21, 512, 0.4, "adam", "f32", "f32", SKIP, None),
-    ("packed_shards_inside_a_tile", 8, 256 * 10, 256, 0.3, "adam", "bf16", "bf16", 0, None),      # pps = 2: four owners per tile
+    ("gather_wide_256", 16, 256 * 61 + 40, 256, 0.1, "adam", "bf16", "bf16", 0, "gather wide packets/tile=8"),
+    ("gather_twin_128_w40", 40, 128 * 90 + 8, 128, 0.1, "sgd", "bf16", "bf16", 0, "gather twin packets/tile=8"),
+    ("gather_twin_512_w3_f32", 3, 512 * 21, 512, 0.4, "adam", "f32", "f32", SKIP, "gather twin packets/tile=2"),
+    ("gather_shards_inside_a_tile", 8, 256 * 10, 256, 0.3, "adam", "bf16", "bf16", 0, "gather wide"),      # pps = 2: four owners per tile
+    ("gather_twin_w2_mixed", 2, 256 * 33 + 24, 256, 0.3, "adam", "bf16", "f32", 0, "gather twin packets/tile=4"),
+    ("packed_wide_256", 16, 256 * 61 + 40, 256, 0.1, "adam", "bf16", "bf16", PACKED, "bulk-copy wide group=8 stale=late packed"),
+    ("packed_twin_128_w40", 40, 128 * 90 + 8, 128, 0.3, "sgd", "bf16", "bf16", PACKED, "bulk-copy twin group=8 stale=late packed"),
+    ("packed_512_w3_f32", 3, 512 * 21, 512, 0.4, "adam", "f32", "f32", SKIP | PACKED, None),
+    ("packed_shards_inside_a_tile", 8, 256 * 10, 256, 0.3, "adam", "bf16", "bf16", PACKED, None),
     ("register_path", 8, 2048 * 9 + 5, 2048, 0.3, "adam", "bf16", "bf16", REG, "register kernel"),
     ("register_small_packets_w17", 17, 264 * 50, 264, 0.2, "adam", "bf16", "f32", 0, "register kernel"),
     ("fewer_packets_than_workers", 8, 3 * 512 - 100, 512, 0.2, "adam", "f32", "bf16", 0, None),
@@ -83,6 +89,7 @@ BAND, POISON = 4096, 0x5A
 
 
 @pytest.mark.parametrize("W,n,P,p,flags", [(8, 2048 * 19 + 1003, 2048, 0.2, 0), (16, 256 * 45 + 40, 256, 0.1, 0),
+                                           (16, 256 * 45 + 40, 256, 0.1, PACKED), (3, 128 * 77 + 8, 128, 0.3, 0),
                                            (64, 1024 * 70 + 16, 1024, 0.3, 0), (8, 2048 * 7 + 5, 2048, 0.3, REG)])
 def test_elided_replicas_between_guard_bands(W, n, P, p, flags):
     """Every replica is exactly lossy_replica_elems long and sits between two poisoned bands: the owner's range
