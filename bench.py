@@ -722,6 +722,7 @@ def main():
     launches0 = L.lossy_kernel_launches(ctx)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
+    torch.cuda.profiler.start()          # a profiler started with --profile-from-start off sees the timed region only
     ev[0].record(stream)
     for i in range(args.steps):
         t += 1
@@ -730,6 +731,7 @@ def main():
     if dist is not None:
         dist.all_reduce(sumsq, op=dist.ReduceOp.SUM)        # the only exchange: W doubles per job
     barrier()
+    torch.cuda.profiler.stop()
     total_ms = ev[0].elapsed_time(ev[-1])
     per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     launches = L.lossy_kernel_launches(ctx) - launches0

@@ -185,8 +185,12 @@ __global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kC
     const uint32_t lgWp = 31u - (uint32_t)__clz((int)Wp);
     const uint32_t Bp = 32u >> lgWp;                        // sub-packets per pass of draws
     const uint32_t wmask = Wp == 32 ? 0xFFFFFFFFu : ((1u << Wp) - 1u);
-    // the old copy of a (replica, sub-packet) pair that misses the broadcast is read by a compute warp several
-    // tiles later for the drift term: start it toward L2 now (one bulk prefetch per pair)
+    // the old copy of a (replica, sub-packet) pair that misses the broadcast is read several tiles later for the
+    // drift term (by a compute warp, or by a replica warp in the RD builds): start it toward L2 now (one bulk
+    // prefetch per pair)
+    // (G.hints bit 2: the host asks for it where few pairs per tile are stale — it gains about 5 % there and
+    // loses as much where they are many: the prefetches then crowd the bulk-copy unit that moves theta, m, v)
+    const bool prefetch_on = kWarpDrift && (G.hints & 4u);
     auto prefetch_stale = [&](uint32_t i, uint32_t j, uint32_t k) {
       bulk_prefetch_l2(reinterpret_cast<const typename RT::raw*>(P.replicas[i]) + rep_index(P, i, j, (uint64_t)k * P.P), P.P * kRB);
     };
@@ -222,9 +226,7 @@ __global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kC
             if (x == ((uint32_t)lane >> lgWp)) st_l = st;
             if ((uint32_t)lane == x) report(q0 + x, j_x, r, st, gbad, pbad);
           }
-          if constexpr (kWarpDrift) {
-            if (sp_l < npk && i_l < W && ((st_l >> i_l) & 1ull)) prefetch_stale(i_l, j_l, k_l);
-          }
+          if (prefetch_on && sp_l < npk && i_l < W && ((st_l >> i_l) & 1ull)) prefetch_stale(i_l, j_l, k_l);
         }
       } else {
         for (uint32_t sp = 0; sp < npk; ++sp) {
@@ -232,7 +234,7 @@ __global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kC
           const uint32_t j_sp = (P.k0 + kfirst + sp) / P.pps;
           packet_masks<AGG | BCAST>(P, kfirst + sp, j_sp, lane, r, st, gbad, pbad);
           if (lane == 0) report(sp, j_sp, r, st, gbad, pbad);
-          if constexpr (kWarpDrift) {
+          if (prefetch_on) {
             for (uint32_t i = lane; i < W; i += 32)
               if ((st >> i) & 1ull) prefetch_stale(i, j_sp, kfirst + sp);
           }

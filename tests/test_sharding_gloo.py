@@ -90,3 +90,47 @@ def test_two_ranks_reproduce_the_single_process_drift():
     want = _run_buckets(_bucket_workloads(), 3)
     assert np.allclose(got, want, rtol=1e-12)
     assert tmax == 2.0
+
+
+def _range_worker(rank, world, port, q):
+    """One bucket in `world` packet ranges with owner-elided replicas: a range holds all, part or none of a
+    worker's shard, and replica i of that range leaves out exactly that part."""
+    from oracle import oracle as O
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = workload.Workload("range_bucket", 5, 512 * 23 + 40, 512, 0.3, "adam", 3e-4, "bf16", "bf16", 3, seed=9)
+    cfg = packet_range_config(w.n, w.packet_elems, rank, world)
+    e0, e1 = cfg["e0"], cfg["e0"] + cfg["n"]
+    o = make_oracle(w, flags=O.REPLICA_SKIP_OWNER, k0=cfg["shard_packet0"], n_slab=cfg["n"], e0=e0)
+    for t in range(1, 4):
+        r = o.step(t, [to_np(workload.grad_slab(w, t, i, e0, e1)) for i in range(w.W)])
+    mine = torch.from_numpy(r["sumsq"].copy())
+    dist.all_reduce(mine, op=dist.ReduceOp.SUM)
+    kept = torch.tensor([float(sum(x.size for x in o.replicas))])
+    dist.all_reduce(kept, op=dist.ReduceOp.SUM)
+    if rank == 0:
+        q.put((mine.numpy(), float(kept)))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_of_packet_ranges_with_owner_elided_replicas():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_range_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got, kept = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = workload.Workload("range_bucket", 5, 512 * 23 + 40, 512, 0.3, "adam", 3e-4, "bf16", "bf16", 3, seed=9)
+    o = make_oracle(w)                                   # the whole bucket, full replicas
+    for t in range(1, 4):
+        r = o.step(t, [to_np(workload.grad_slab(w, t, i, 0, w.n)) for i in range(w.W)])
+    assert np.allclose(got, r["sumsq"], rtol=1e-12) and got.max() > 0
+    assert kept == (w.W - 1) * w.n                       # every element is stored W - 1 times over the ranks
