@@ -307,7 +307,7 @@ bool gather_geometry(const lossy_ctx* ctx, bool drift, TmaGeom& G) {
   G.stage_bytes = (G.grad_slots * kTile * gb + 3 * kTile * 4 + 127u) & ~127u;
   // fp64 drift sums per compute warp and replica, the wire ring, and (few workers, drift norms) the replica warps' scratch
   G.state_bytes = CW * kMaxW * (uint32_t)sizeof(double) + kWireRing * kTile * rb;
-  if (drift && gather_rd<CW>(c)) G.state_bytes += GatherShape<CW>::kReplicaWarps * 2u * rd_buffer_bytes<CW>(rb);
+  if (drift && gather_rd<CW>(c)) G.state_bytes += GatherShape<CW, true>::kReplicaWarps * 2u * rd_buffer_bytes<CW>(rb);
   const uint32_t budget = (227u * 1024u) / GatherShape<CW>::kCtasPerSm - 1024u;
   const uint32_t avail = (uint32_t)ctx->smem_optin < budget ? (uint32_t)ctx->smem_optin : budget;
   if (avail < kGatherSmemFixed + G.state_bytes + 2 * G.stage_bytes) return false;
@@ -342,7 +342,7 @@ int launch_gather(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStream_
       if (ctx->device < kMaxDevices) opted_in[ctx->device] = true;
     }
   }
-  kern<<<blocks, GatherShape<CW>::kThreads, smem, s>>>(P, G);
+  kern<<<blocks, GatherShape<CW, RD>::kThreads, smem, s>>>(P, G);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail_cuda(ctx, "gather kernel launch", e);
   ctx->launches++;

@@ -28,9 +28,10 @@ namespace lossy {
 
 constexpr uint32_t kGatherRing = 8;     // tiles whose masks may be published ahead of the replica warps
 constexpr uint32_t kWireRing = 4;       // wire tiles between the compute warps and the replica warps
-template <int CW> struct GatherShape {
+// RD: the build in which the replica warps also read the stale copies (see the kernel): one replica per warp
+template <int CW, bool RD = false> struct GatherShape {
   static constexpr int kProducers = CW >= 16 ? 2 : 1;                     // gather warps
-  static constexpr int kReplicaWarps = CW >= 16 ? 4 : 2;
+  static constexpr int kReplicaWarps = (CW >= 16 || RD) ? 4 : 2;
   static constexpr int kThreads = (CW + 2 + kProducers + kReplicaWarps) * 32;   // compute + mask + gather + store + replica
   static constexpr int kTile = CW * 32 * kEpl;
   static constexpr int kCtasPerSm = CW >= 16 ? 1 : 2;
@@ -38,8 +39,8 @@ template <int CW> struct GatherShape {
 constexpr uint32_t kRdMaxWorkers = 4;   // RD builds (below) serve at most this many workers
 // RD builds: bytes of one scratch buffer of a replica warp = the rows of all the replicas it can own
 template <int CW> __host__ __device__ constexpr uint32_t rd_buffer_bytes(uint32_t replica_elem_bytes) {
-  return ((kRdMaxWorkers + GatherShape<CW>::kReplicaWarps - 1u) / GatherShape<CW>::kReplicaWarps) *
-         (uint32_t)GatherShape<CW>::kTile * replica_elem_bytes;
+  return ((kRdMaxWorkers + GatherShape<CW, true>::kReplicaWarps - 1u) / GatherShape<CW, true>::kReplicaWarps) *
+         (uint32_t)GatherShape<CW, true>::kTile * replica_elem_bytes;
 }
 constexpr uint32_t kGatherMaxStages = 8;    // a tile of few workers is small: more of them in flight
 constexpr uint32_t kGatherBarBytes = 512;   // 3 barriers per stage, 2 per mask-ring and wire-ring entry (8 B each), the abort flag
@@ -117,13 +118,13 @@ __device__ __forceinline__ void finish_tile_lane(const Params& P, float (&acc)[k
 // neither their instruction budget nor the tile's duration hides those loads; with many replicas the scratch
 // would not fit and the sixteen compute warps' early requests hide them better.
 template <class GT, class RT, int OPT, bool DRIFTK, int CW, bool RD = false>
-__global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kCtasPerSm)
+__global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW, RD>::kCtasPerSm)
     lossy_fused_gather_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
   static_assert(!RD || DRIFTK, "RD is a way of computing the drift norms");
   constexpr bool kWarpDrift = DRIFTK && !RD;               // the compute warps read the stale copies
-  constexpr int kTile = GatherShape<CW>::kTile;
-  constexpr int kNP = GatherShape<CW>::kProducers;
-  constexpr int kNR = GatherShape<CW>::kReplicaWarps;
+  constexpr int kTile = GatherShape<CW, RD>::kTile;
+  constexpr int kNP = GatherShape<CW, RD>::kProducers;
+  constexpr int kNR = GatherShape<CW, RD>::kReplicaWarps;
   constexpr int kGroup = 8;
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
   constexpr uint32_t kRowG = kTile * kGB, kRowR = kTile * kRB;          // bytes of one worker's / replica's row of a tile
@@ -357,7 +358,7 @@ __global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kC
         const uint32_t live = __ballot_sync(0xFFFFFFFFu, (stale_l >> i) & 1ull) & 0xFFu & live_tile;
         if (live == 0u) continue;
         const unsigned char* base = reinterpret_cast<const unsigned char*>(P.replicas[i]);
-        float sq = 0.0f;
+        float2 sq2 = make_float2(0.0f, 0.0f);                                 // two running sums (packed fp32 pairs of sm_100)
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
           const uint32_t el0 = (uint32_t)c * kElemsPerChunk;                    // the chunk's sub-packets, as bits
@@ -375,22 +376,25 @@ __global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kC
             const uint4 ov = *reinterpret_cast<const uint4*>(sc);               // each lane reads back what it copied itself
             const uint4 wv = *reinterpret_cast<const uint4*>(wt + off);
             const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w}, ww[4] = {wv.x, wv.y, wv.z, wv.w};
+            if constexpr (RT::kVecs == 2) {                // fp32 replicas: one element per word
 #pragma unroll
-            for (int h = 0; h < 4; ++h) {
-              if constexpr (RT::kVecs == 2) {              // fp32 replicas: one element per word
-                const float d0 = __fsub_rn(__uint_as_float(ow[h]), __uint_as_float(ww[h]));
-                sq = __fadd_rn(sq, __fmul_rn(d0, d0));
-              } else {                                      // bf16 replicas: two elements per word
-                const float d0 = __fsub_rn(__uint_as_float(ow[h] << 16), __uint_as_float(ww[h] << 16));
-                const float d1 = __fsub_rn(__uint_as_float(ow[h] & 0xFFFF0000u), __uint_as_float(ww[h] & 0xFFFF0000u));
-                sq = __fadd_rn(sq, __fmul_rn(d0, d0));
-                sq = __fadd_rn(sq, __fmul_rn(d1, d1));
+              for (int h = 0; h < 4; h += 2) {
+                const float2 d = __fadd2_rn(make_float2(__uint_as_float(ow[h]), __uint_as_float(ow[h + 1])),
+                                            make_float2(-__uint_as_float(ww[h]), -__uint_as_float(ww[h + 1])));
+                sq2 = __fadd2_rn(sq2, __fmul2_rn(d, d));
+              }
+            } else {                                        // bf16 replicas: two elements per word
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const float2 d = __fadd2_rn(make_float2(__uint_as_float(ow[h] << 16), __uint_as_float(ow[h] & 0xFFFF0000u)),
+                                            make_float2(-__uint_as_float(ww[h] << 16), -__uint_as_float(ww[h] & 0xFFFF0000u)));
+                sq2 = __fadd2_rn(sq2, __fmul2_rn(d, d));
               }
             }
           }
         }
         if (pass == 1) {
-          const float tot = warp_sum(sq);
+          const float tot = warp_sum(__fadd_rn(sq2.x, sq2.y));
           if (lane == 0) warp_acc[i] += (double)tot;        // row 0 of the sums: one accumulator per replica
         }
       }
@@ -595,7 +599,7 @@ __global__ void __launch_bounds__(GatherShape<CW>::kThreads, GatherShape<CW>::kC
       for (int w = 0; w < CW; ++w) t += warp_acc[w * kMaxW + threadIdx.x];
       P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
     }
-    if (P.ticket) drift_last_block(P, warp, lane, GatherShape<CW>::kThreads / 32);
+    if (P.ticket) drift_last_block(P, warp, lane, GatherShape<CW, RD>::kThreads / 32);
   }
 }
 
