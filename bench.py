@@ -612,6 +612,7 @@ def main():
                     help="single process: run only packet range R of G of the bucket (what rank R of a G-GPU --strong job runs)")
     ap.add_argument("--register-path", action="store_true", help="time the register-path kernel, not the bulk-copy pipeline")
     ap.add_argument("--skip-owner", action="store_true", help="headline with owner-elided replicas (LOSSY_REPLICA_SKIP_OWNER)")
+    ap.add_argument("--gather-path", action="store_true", help="small packets: force the gather pipeline (LOSSY_GATHER_PATH)")
     ap.add_argument("--e2e-steps", type=int, default=-1, help="steps of the host-buffer leg (default: min(steps, 10))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-timed-region", action="store_true",
@@ -684,7 +685,8 @@ def main():
         w = workload.scaled(w, w.n, packet_base=rank * w.K, seed=w.seed)
     gdt, rdt = tdt(w.grad_dtype), tdt(w.replica_dtype)
     adam = w.optimizer == "adam"
-    flags = (L.LOSSY_REGISTER_PATH if args.register_path else 0) | (L.LOSSY_REPLICA_SKIP_OWNER if args.skip_owner else 0)
+    flags = ((L.LOSSY_REGISTER_PATH if args.register_path else 0) | (L.LOSSY_REPLICA_SKIP_OWNER if args.skip_owner else 0)
+             | (L.LOSSY_GATHER_PATH if args.gather_path else 0))
     ctx = make_ctx(L, w, flags, **rng_kw)
     plan = L.lossy_describe_plan(ctx, True)       # the build the library's launch policy picks for this workload
     master = workload.theta0_slab(w, e_off, e_off + w.n, dev)

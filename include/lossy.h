@@ -87,7 +87,10 @@ enum {
   /* Packets shorter than a tile of the fused step: use the packed bulk-copy build (one bulk copy per worker and
    * tile, dropped sub-packets fetched too) where the launch policy allows it, instead of the gather pipeline
    * (per-lane asynchronous copies of the delivered sub-packets only). Same results; for comparison and tests. */
-  LOSSY_PACKED_BULK = 16u
+  LOSSY_PACKED_BULK = 16u,
+  /* Packets shorter than a tile: use the gather pipeline wherever one of its builds fits, also where the launch
+   * policy would pick the register kernel (many workers at high loss). Same results; for comparison and tests. */
+  LOSSY_GATHER_PATH = 32u
 };
 
 #define LOSSY_MAX_WORKERS 64u
@@ -103,7 +106,7 @@ typedef struct {
   uint32_t grad_dtype;   /* LOSSY_F32 or LOSSY_BF16                                     */
   uint32_t replica_dtype;/* LOSSY_F32 or LOSSY_BF16 (bf16 = round-to-nearest-even cast) */
   uint32_t optimizer;    /* LOSSY_SGD or LOSSY_ADAM                                     */
-  uint32_t flags;        /* OR of LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH, LOSSY_REPLICA_SKIP_OWNER */
+  uint32_t flags;        /* OR of the LOSSY_* flags above */
   float lr, beta1, beta2, eps; /* eta_t and Adam's constants (beta/eps unused for SGD)  */
   /* Packet-range sharding (several GPUs simulate one bucket, each a contiguous range of its
    * packets for all W workers): this context's packet 0 is packet shard_packet0 of a bucket of

@@ -18,6 +18,7 @@ LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE, LOSSY_ELIMIT =
 LOSSY_F32, LOSSY_BF16 = 0, 1
 LOSSY_SGD, LOSSY_ADAM = 0, 1
 LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH, LOSSY_REPLICA_SKIP_OWNER, LOSSY_PACKED_BULK = 1, 2, 4, 8, 16
+LOSSY_GATHER_PATH = 32
 
 EXPORTS = [
     "lossy_init", "lossy_destroy", "lossy_set_lr", "lossy_set_bursty", "lossy_set_reliable", "lossy_packet_sqnorms", "lossy_aggregate", "lossy_step", "lossy_broadcast",

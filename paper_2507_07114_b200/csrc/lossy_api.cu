@@ -389,7 +389,7 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
     // packet allows it (256 elements and up).
     const lossy_config& c = ctx->cfg;
     const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
-    const bool reg_ahead = (c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15);
+    const bool reg_ahead = !(c.flags & LOSSY_GATHER_PATH) && ((c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15));
     if (!reg_ahead) {
       int rc = LOSSY_OK;
       if (c.W > kRdMaxWorkers) rc = try_gather<16>(ctx, P, drift, s, blocks, used);
@@ -637,7 +637,7 @@ int lossy_init(const lossy_config* cfg, lossy_ctx** out) {
   if (cfg->packet_elems == 0 || cfg->packet_elems % 8 != 0) return LOSSY_EINVAL;
   if (!(cfg->p_grad >= 0.0 && cfg->p_grad < 1.0) || !(cfg->p_param >= 0.0 && cfg->p_param < 1.0)) return LOSSY_EINVAL;
   if (cfg->grad_dtype > LOSSY_BF16 || cfg->replica_dtype > LOSSY_BF16 || cfg->optimizer > LOSSY_ADAM) return LOSSY_EINVAL;
-  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH | LOSSY_REPLICA_SKIP_OWNER | LOSSY_PACKED_BULK))
+  if (cfg->flags & ~(uint32_t)(LOSSY_SELF_LOSSLESS | LOSSY_ZERO_SKIP | LOSSY_REGISTER_PATH | LOSSY_REPLICA_SKIP_OWNER | LOSSY_PACKED_BULK | LOSSY_GATHER_PATH))
     return LOSSY_EINVAL;
   const uint64_t K = (cfg->n + cfg->packet_elems - 1) / cfg->packet_elems;
   const uint64_t cpp = (cfg->packet_elems + kChunk - 1) / kChunk;

@@ -199,7 +199,7 @@ def run_parity(w: workload.Workload, steps, *, fused=True, flags=0, p_grad=None,
                alg1=False, burst=None):
     """Element-by-element parity of a whole (small) run. Returns the GpuRun for further checks."""
     gpu = GpuRun(w, flags=flags, p_grad=p_grad, p_param=p_param, alg1=alg1, burst=burst)
-    orc = make_oracle(w, flags=flags & ~(L.LOSSY_REGISTER_PATH | L.LOSSY_PACKED_BULK), p_grad=p_grad, p_param=p_param, alg1=alg1,
+    orc = make_oracle(w, flags=flags & ~(L.LOSSY_REGISTER_PATH | L.LOSSY_PACKED_BULK | L.LOSSY_GATHER_PATH), p_grad=p_grad, p_param=p_param, alg1=alg1,
                       burst=burst)                                                  # those bits only pick the kernel
     for t in range(1, steps + 1):
         gs = [workload.grad_slab(w, t, i, 0, w.n) for i in range(w.W)]

@@ -103,6 +103,9 @@ EDGE = [
     ("packed_twin_w24_two_per_tile", 24, 512 * 45 + 8, 512, 0.05, "sgd", "bf16", "bf16", 0),
     ("packed_128_elements_any_loss", 40, 128 * 90, 128, 0.4, "adam", "bf16", "f32", LOSSLESS),
     ("packed_128_w4", 4, 128 * 33 + 16, 128, 0.1, "sgd", "f32", "bf16", 0),
+    # the gather pipeline where the policy would pick the register kernel: many stale copies per sub-packet
+    ("gather_forced_w24_high_loss", 24, 256 * 70 + 8, 256, 0.4, "adam", "bf16", "bf16", L.LOSSY_GATHER_PATH),
+    ("gather_forced_w64_f32_replicas", 64, 512 * 33, 512, 0.3, "sgd", "bf16", "f32", L.LOSSY_GATHER_PATH),
 ]
 
 
@@ -196,7 +199,7 @@ def test_empty_bucket_is_a_noop_and_bad_arguments_are_rejected():
     assert L.lossy_kernel_launches(ctx) == 0
     L.lossy_destroy(ctx)
     for bad in (dict(W=0), dict(W=65), dict(packet_elems=0), dict(packet_elems=12), dict(p_grad=1.0),
-                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=32), dict(optimizer=5)):
+                dict(p_param=-0.1), dict(p_grad=float("nan")), dict(flags=64), dict(optimizer=5)):
         kw = dict(W=2, n=64, packet_elems=64, p_grad=0.1, p_param=0.1, seed=0, grad_dtype=torch.float32,
                   replica_dtype=torch.float32, optimizer="sgd", lr=0.1)
         kw.update(bad)

@@ -70,7 +70,7 @@ def test_configuration_is_validated_on_the_host_before_any_cuda_call():
                 lr=3e-4, beta1=0.9, beta2=0.95, eps=1e-8, shard_packet0=0, bucket_packets=0)
     bad = [dict(W=0), dict(W=65), dict(packet_elems=0), dict(packet_elems=100), dict(p_grad=1.0),
            dict(p_param=-1e-9), dict(p_grad=float("nan")), dict(grad_dtype=2), dict(replica_dtype=7),
-           dict(optimizer=2), dict(flags=64), dict(n=2 ** 40, packet_elems=8),          # more than 2^31 chunks
+           dict(optimizer=2), dict(flags=128), dict(n=2 ** 40, packet_elems=8),          # more than 2^31 chunks
            dict(shard_packet0=1), dict(shard_packet0=8, bucket_packets=12),             # range leaves the bucket
            dict(n=2048 * 10 - 8, bucket_packets=20)]                                    # ragged range inside a bucket
     for change in bad:
