@@ -284,12 +284,10 @@ int try_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
 // barriers, the ring of tile masks, stage headers; the drift sums per compute warp, the wire ring and the stages follow
 constexpr uint32_t kGatherSmemFixed = kGatherBarBytes + kGatherRing * sizeof(TileMasks) + kGatherMaxStages * sizeof(StageHdr);
 
-// few workers (twin geometry): the replica warps read the stale copies for the drift norms
+// rd: the stale copies are read outside the compute warps (twin geometry: by the replica warps, one replica each;
+// wide geometry: by drift warps of their own)
 template <int CW>
-bool gather_rd(const lossy_config& c) { return CW == 8 && c.W <= kRdMaxWorkers; }
-
-template <int CW>
-bool gather_geometry(const lossy_ctx* ctx, bool drift, TmaGeom& G) {
+bool gather_geometry(const lossy_ctx* ctx, bool rd, TmaGeom& G) {
   constexpr uint32_t kTile = GatherShape<CW>::kTile;
   const lossy_config& c = ctx->cfg;
   const uint64_t kfull = c.n / c.packet_elems;               // packets that are complete
@@ -305,14 +303,43 @@ bool gather_geometry(const lossy_ctx* ctx, bool drift, TmaGeom& G) {
   G.groups = (c.W + 7u) / 8u;
   // a stage holds the group's gradient rows and theta, m, v
   G.stage_bytes = (G.grad_slots * kTile * gb + 3 * kTile * 4 + 127u) & ~127u;
-  // fp64 drift sums per compute warp and replica, the wire ring, and (few workers, drift norms) the replica warps' scratch
-  G.state_bytes = CW * kMaxW * (uint32_t)sizeof(double) + kWireRing * kTile * rb;
-  if (drift && gather_rd<CW>(c)) G.state_bytes += GatherShape<CW, true>::kReplicaWarps * 2u * rd_buffer_bytes<CW>(rb);
+  // fp64 drift sums per adding warp and replica, the wire ring, and (rd) the scratch for the stale copies
+  G.state_bytes = (uint32_t)(rd ? GatherShape<CW, true>::kAccRows : CW) * kMaxW * (uint32_t)sizeof(double) + kWireRing * kTile * rb;
+  const uint32_t row_chunks = kTile * rb / 512u;             // 512-byte chunks of one replica's row of a tile
+  uint32_t scratch_unit = 0;                                  // bytes of scratch per chunk of capacity
+  if (rd) {
+    using Shape = GatherShape<CW, true>;
+    scratch_unit = (uint32_t)(Shape::kDriftWarps ? Shape::kDriftWarps : Shape::kReplicaWarps) * Shape::kRdBuffers * 512u;
+    // twin: a replica warp owns one replica, its whole row fits; wide: at least four chunks per drift warp, more below
+    G.rd_cap = Shape::kDriftWarps ? 4u : row_chunks;
+    G.state_bytes += G.rd_cap * scratch_unit;
+  }
   const uint32_t budget = (227u * 1024u) / GatherShape<CW>::kCtasPerSm - 1024u;
   const uint32_t avail = (uint32_t)ctx->smem_optin < budget ? (uint32_t)ctx->smem_optin : budget;
   if (avail < kGatherSmemFixed + G.state_bytes + 2 * G.stage_bytes) return false;
   G.stages = (avail - kGatherSmemFixed - G.state_bytes) / G.stage_bytes;
   if (G.stages > 4u) G.stages = 4u;                           // more measured no faster (W = 2..32)
+  if (rd && GatherShape<CW, true>::kDriftWarps) {
+    // wide: what the stages leave goes to the scratch, up to every chunk of a drift warp's replicas
+    const uint32_t left = avail - kGatherSmemFixed - G.state_bytes - G.stages * G.stage_bytes;
+    // a replica's row in 2^lgsplit parts, W * 2^lgsplit parts dealt round robin: the fewest parts that balance the drift warps
+    const uint32_t nd = GatherShape<CW, true>::kDriftWarps;
+    // (a warp's cost: its share of a row, plus about a sixteenth of a row per part whatever the part holds: W = 17 in 8
+    // parts per row, 17 parts per warp, ran at 0.56 where W = 16 in whole rows, 2 per warp, ran at 0.85; W = 12 in
+    // halves 0.79 against 0.74 in whole rows; W = 5, P = 512 in quarters 0.86 against 0.83)
+    uint32_t best = ~0u, share = 8u;
+    for (uint32_t lg = 0; (1u << lg) <= G.packets_per_tile && lg <= 2u; ++lg) {
+      const uint32_t parts = ((c.W << lg) + nd - 1u) / nd;                   // a warp's parts ...
+      const uint32_t eighths = parts * (8u >> lg);                            // ... and its share in eighths of a row
+      const uint32_t cost = 2u * eighths + parts;
+      if (cost < best) { best = cost; share = eighths; G.rd_lgsplit = lg; }
+    }
+    const uint32_t most = (share * row_chunks + 7u) / 8u;
+    uint32_t more = left / scratch_unit;
+    if (G.rd_cap + more > most) more = most > G.rd_cap ? most - G.rd_cap : 0u;
+    G.rd_cap += more;
+    G.state_bytes += more * scratch_unit;
+  }
   G.tiles_per_packet = 1;
   const uint64_t tiles = (kfull + G.packets_per_tile - 1) / G.packets_per_tile;
   if (tiles >= (1ull << 31)) return false;
@@ -361,15 +388,14 @@ int dispatch_gather(lossy_ctx* ctx, const Params& P, const TmaGeom& G, cudaStrea
 }
 
 template <int CW>
-int try_gather(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_t* blocks, bool* used) {
+int try_gather(lossy_ctx* ctx, const Params& P, bool drift, bool rd, cudaStream_t s, uint32_t* blocks, bool* used) {
   TmaGeom G = {};
-  if (!gather_geometry<CW>(ctx, drift, G)) return LOSSY_OK;
+  if (!gather_geometry<CW>(ctx, drift && rd, G)) return LOSSY_OK;
   *used = true;
   if (ctx->plan)
-    snprintf(ctx->plan, ctx->plan_size, "gather %s packets/tile=%u stages=%u", CW == 16 ? "wide" : "twin", G.packets_per_tile, G.stages);
-  if constexpr (CW == 8) {
-    if (drift && gather_rd<CW>(ctx->cfg)) return dispatch_gather<true, CW, true>(ctx, P, G, s, blocks);
-  }
+    snprintf(ctx->plan, ctx->plan_size, "gather %s packets/tile=%u stages=%u%s", CW == 16 ? "wide" : "twin", G.packets_per_tile, G.stages,
+             drift && rd && CW == 16 ? " drift-warps" : "");
+  if (drift && rd) return dispatch_gather<true, CW, true>(ctx, P, G, s, blocks);
   return drift ? dispatch_gather<true, CW, false>(ctx, P, G, s, blocks) : dispatch_gather<false, CW, false>(ctx, P, G, s, blocks);
 }
 
@@ -381,20 +407,27 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   const TmaPolicy t = tma_policy(ctx->cfg);
   if (!(ctx->cfg.flags & LOSSY_PACKED_BULK) && ctx->cfg.packet_elems < (uint32_t)TmaShape<8>::kTile) {
     // Packets shorter than a tile (128, 256 or 512 elements): the gather pipeline, where it beats the register
-    // kernel (fractions of the copy rate at 256 elements, W = 6..64): up to eight workers at every loss rate
-    // (0.72-0.98 against 0.60-0.92 for the packed bulk-copy build); more workers up to moderate loss
-    // (p = 0.05: 0.91-0.98 against 0.89-0.93); at high loss with many workers the register kernel stays ahead
-    // (p = 0.3, W >= 12: 0.71-0.77 against 0.65-0.77; p = 0.2, W = 32: 0.85 against 0.79). Few workers (W <= 4)
-    // run the twin geometry, whose replica warps also read the stale copies; the rest the wide one, where a
-    // packet allows it (256 elements and up).
+    // kernel (fractions of the copy rate, 20 steps of a 202 M element bucket).
+    //  * 4..24 workers, packets of 256 or 512 elements, fewer than 7.5 stale replicas per sub-packet: the wide
+    //    geometry with drift warps of its own (W = 16, P = 256: 1.00 / 0.96 / 0.94 / 0.90 / 0.85 at p = 0 / 0.05 /
+    //    0.1 / 0.2 / 0.3, where the compute warps' reads gave 0.94 / 0.94 / 0.96 / 0.81 / 0.70 and the register
+    //    kernel 0.91 / 0.84 / 0.82 / 0.79 / 0.76; W = 8: 0.97 and 0.84 at p = 0.1 and 0.3 against 0.91 and 0.78;
+    //    W = 24, p = 0.3: 0.81 against 0.72; W = 4: 0.80-0.83 against 0.75-0.81 for the twin geometry);
+    //  * beyond that the drift warps fall behind (W = 17, p = 0.5: 0.43): many workers at high loss stay with the
+    //    register kernel (p = 0.3, W >= 12: 0.71-0.77 against 0.65-0.77; p = 0.2, W = 32: 0.85 against 0.79-0.84),
+    //    the rest with the compute warps' reads (W = 32, p = 0.05: 0.96 against 0.91; W = 64, p = 0.1: 0.89);
+    //  * two or three workers, and packets of 128 elements: the twin geometry (W = 2: 0.78-0.81 against 0.69-0.74
+    //    for the wide one), whose replica warps also read the stale copies up to four workers.
     const lossy_config& c = ctx->cfg;
     const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
-    const bool reg_ahead = !(c.flags & LOSSY_GATHER_PATH) && ((c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15));
+    const bool wide_fits = c.packet_elems * (uint32_t)kMaxSub >= (uint32_t)GatherShape<16>::kTile;
+    const bool drift_warps = wide_fits && c.W >= 4u && c.W <= 24u && (c.W - 1u) * c.p_param < 7.5;
+    const bool reg_ahead = !(c.flags & LOSSY_GATHER_PATH) && !drift_warps && ((c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15));
     if (!reg_ahead) {
       int rc = LOSSY_OK;
-      if (c.W > kRdMaxWorkers) rc = try_gather<16>(ctx, P, drift, s, blocks, used);
+      if (c.W >= 4u) rc = try_gather<16>(ctx, P, drift, drift_warps, s, blocks, used);
       if (rc || *used) return rc;
-      rc = try_gather<8>(ctx, P, drift, s, blocks, used);
+      rc = try_gather<8>(ctx, P, drift, c.W <= kRdTwinMaxWorkers, s, blocks, used);
       if (rc || *used) return rc;
     }
   }

@@ -28,20 +28,19 @@ namespace lossy {
 
 constexpr uint32_t kGatherRing = 8;     // tiles whose masks may be published ahead of the replica warps
 constexpr uint32_t kWireRing = 4;       // wire tiles between the compute warps and the replica warps
-// RD: the build in which the replica warps also read the stale copies (see the kernel): one replica per warp
+// RD: the build in which the stale copies are read outside the compute warps (see the kernel): by the replica
+// warps in the twin geometry, by drift warps of their own in the wide one
 template <int CW, bool RD = false> struct GatherShape {
   static constexpr int kProducers = CW >= 16 ? 2 : 1;                     // gather warps
   static constexpr int kReplicaWarps = (CW >= 16 || RD) ? 4 : 2;
-  static constexpr int kThreads = (CW + 2 + kProducers + kReplicaWarps) * 32;   // compute + mask + gather + store + replica
+  static constexpr int kDriftWarps = (CW >= 16 && RD) ? 8 : 0;
+  static constexpr int kRdBuffers = kDriftWarps ? 1 : 2;                  // scratch buffers per warp that reads stale copies
+  static constexpr int kAccRows = RD ? (kDriftWarps ? kMaxSub : 1) : CW;  // rows of fp64 drift sums: per compute warp, or per part of a row (RD)
+  static constexpr int kThreads = (CW + 2 + kProducers + kReplicaWarps + kDriftWarps) * 32;   // compute + mask + gather + store + replica (+ drift)
   static constexpr int kTile = CW * 32 * kEpl;
   static constexpr int kCtasPerSm = CW >= 16 ? 1 : 2;
 };
-constexpr uint32_t kRdMaxWorkers = 4;   // RD builds (below) serve at most this many workers
-// RD builds: bytes of one scratch buffer of a replica warp = the rows of all the replicas it can own
-template <int CW> __host__ __device__ constexpr uint32_t rd_buffer_bytes(uint32_t replica_elem_bytes) {
-  return ((kRdMaxWorkers + GatherShape<CW, true>::kReplicaWarps - 1u) / GatherShape<CW, true>::kReplicaWarps) *
-         (uint32_t)GatherShape<CW, true>::kTile * replica_elem_bytes;
-}
+constexpr uint32_t kRdTwinMaxWorkers = 4;   // twin RD builds serve at most this many workers: one replica per replica warp
 constexpr uint32_t kGatherMaxStages = 8;    // a tile of few workers is small: more of them in flight
 constexpr uint32_t kGatherBarBytes = 512;   // 3 barriers per stage, 2 per mask-ring and wire-ring entry (8 B each), the abort flag
 static_assert((3 * kGatherMaxStages + 2 * kGatherRing + 2 * kWireRing) * 8 + 4 <= kGatherBarBytes, "barrier area too small");
@@ -112,11 +111,12 @@ __device__ __forceinline__ void finish_tile_lane(const Params& P, float (&acc)[k
   }
 }
 
-// RD (drift norms with few replicas): the replica warps, not the compute warps, read the old copies of the
-// stale (replica, sub-packet) pairs — with asynchronous copies into a double-buffered scratch, requested one
-// tile ahead. With few workers the compute warps are bound by their issue slots and a tile is short, so that
-// neither their instruction budget nor the tile's duration hides those loads; with many replicas the scratch
-// would not fit and the sixteen compute warps' early requests hide them better.
+// RD (a way of computing the drift norms): the old copies of the stale (replica, sub-packet) pairs are read outside
+// the compute warps, with asynchronous copies into a scratch of G.rd_cap 512-byte chunks per buffer, requested as
+// soon as the tile's masks are known and used once its wire tile exists; chunks beyond the scratch are loaded
+// directly. Twin geometry (few workers): the replica warps do it, one tile ahead in the second of two buffers.
+// Wide geometry: four drift warps of their own do nothing else; one buffer is enough, because the masks run
+// several tiles ahead of the wire tile.
 template <class GT, class RT, int OPT, bool DRIFTK, int CW, bool RD = false>
 __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW, RD>::kCtasPerSm)
     lossy_fused_gather_kernel(const __grid_constant__ Params P, const __grid_constant__ TmaGeom G) {
@@ -125,6 +125,8 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
   constexpr int kTile = GatherShape<CW, RD>::kTile;
   constexpr int kNP = GatherShape<CW, RD>::kProducers;
   constexpr int kNR = GatherShape<CW, RD>::kReplicaWarps;
+  constexpr int kND = GatherShape<CW, RD>::kDriftWarps;
+  constexpr int kAccRows = GatherShape<CW, RD>::kAccRows;
   constexpr int kGroup = 8;
   constexpr uint32_t kGB = sizeof(typename GT::raw), kRB = sizeof(typename RT::raw);
   constexpr uint32_t kRowG = kTile * kGB, kRowR = kTile * kRB;          // bytes of one worker's / replica's row of a tile
@@ -136,10 +138,10 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
   TileMasks* ring = reinterpret_cast<TileMasks*>(smem + kGatherBarBytes);
   StageHdr* hdrs = reinterpret_cast<StageHdr*>(smem + kGatherBarBytes + kGatherRing * sizeof(TileMasks));
   double* warp_acc = reinterpret_cast<double*>(smem + kGatherBarBytes + kGatherRing * sizeof(TileMasks) + kGatherMaxStages * sizeof(StageHdr));
-  unsigned char* wring = reinterpret_cast<unsigned char*>(warp_acc + CW * kMaxW);
-  constexpr uint32_t kRdBuf = rd_buffer_bytes<CW>(kRB);
-  unsigned char* rscratch = wring + kWireRing * kRowR;     // RD: two buffers per replica warp
-  unsigned char* stage0 = rscratch + (RD ? kNR * 2u * kRdBuf : 0u);
+  unsigned char* wring = reinterpret_cast<unsigned char*>(warp_acc + kAccRows * kMaxW);
+  const uint32_t rd_buf = G.rd_cap * 512u;                 // RD: bytes of one scratch buffer
+  unsigned char* rscratch = wring + kWireRing * kRowR;     // RD: kRdBuffers buffers per warp that reads stale copies
+  unsigned char* stage0 = rscratch + (RD ? (uint32_t)(kND ? kND : kNR) * GatherShape<CW, RD>::kRdBuffers * rd_buf : 0u);
   const uint32_t S = G.stages;
   const uint32_t off_th = G.grad_slots * kRowG;
   const uint32_t off_m = off_th + kTile * 4, off_v = off_m + kTile * 4;
@@ -156,7 +158,7 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
   auto wfull_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kGatherMaxStages + 2 * kGatherRing + q]); };
   auto wempty_bar = [&](uint32_t q) { return smem_u32(&bars[3 * kGatherMaxStages + 2 * kGatherRing + kWireRing + q]); };
 
-  for (uint32_t q = threadIdx.x; q < (uint32_t)CW * kMaxW; q += blockDim.x) warp_acc[q] = 0.0;
+  for (uint32_t q = threadIdx.x; q < (uint32_t)kAccRows * kMaxW; q += blockDim.x) warp_acc[q] = 0.0;
   if (threadIdx.x == 0) {
     *abort_flag = 0u;
     for (uint32_t s = 0; s < S; ++s) {
@@ -166,17 +168,91 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
     }
     for (uint32_t q = 0; q < kGatherRing; ++q) {
       mbar_init(mfull_bar(q), 1);
-      mbar_init(mempty_bar(q), kNR);                 // the replica warps are the last readers of a tile's masks
+      mbar_init(mempty_bar(q), kNR + kND);           // the replica (and drift) warps are the last readers of a tile's masks
     }
     for (uint32_t q = 0; q < kWireRing; ++q) {
       mbar_init(wfull_bar(q), CW);
-      mbar_init(wempty_bar(q), kNR);
+      mbar_init(wempty_bar(q), kNR + kND);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
   }
   __syncthreads();
 
+  constexpr int kChunks = kRowR / 512u;                     // a replica's row of a tile in 512-byte chunks
+  constexpr uint32_t kElemsPerChunk = 512u / kRB;
+  // Wide RD builds. A replica's row of a tile is cut into 2^lgf parts (the host balances the W * 2^lgf parts over
+  // the drift warps); a warp takes parts first, first + stride, ... PASS 0 requests the old copies of their stale
+  // (replica, sub-packet) pairs into `buffer`, chunk after chunk in the order (part, chunk); pass 1 takes their
+  // squared differences against the wire tile: fp32 per lane within a part's chunks, one warp reduction per part
+  // and tile, fp64 from there on (each (replica, part) has one accumulator, touched by one warp alone, in tile
+  // order; the CTA's exit adds a replica's parts in ascending order).
+  // One warp runs this alone, so its instructions are fetched for it alone: the walk visits the stale chunks only
+  // and is kept short (one loop body for both passes, nothing unrolled), and each role calls it from one place.
+  constexpr uint32_t kLgEpc = kElemsPerChunk == 256u ? 8u : 7u;
+  auto drift_pass = [&](const TileMasks& tm, uint32_t first, uint32_t stride, unsigned char* buffer, int pass, const unsigned char* wt) {
+    const uint32_t lgf = G.rd_lgsplit, part = G.packets_per_tile >> lgf;   // a replica's row in 2^lgf parts of `part` sub-packets
+    const uint64_t stale_l = tm.stale[lane & (kMaxSub - 1)];
+    const uint32_t j_l = tm.j[lane & (kMaxSub - 1)];
+    const uint32_t live_tile = (1u << tm.npk) - 1u;       // entries behind a short last tile are marked stale everywhere
+    const uint64_t e0 = tm.e0;
+    const bool whole = lgP >= kLgEpc;                      // a sub-packet is one or more whole chunks (else a chunk holds several)
+    const uint32_t sh = whole ? lgP - kLgEpc : kLgEpc - lgP;
+    uint32_t n = 0;                                        // stale chunks met so far (warp-uniform)
+#pragma unroll 1
+    for (uint32_t u = first; u < (W << lgf); u += stride) {
+      const uint32_t i = u >> lgf, h = u & ((1u << lgf) - 1u);
+      const uint32_t live = __ballot_sync(0xFFFFFFFFu, (stale_l >> i) & 1ull) & live_tile & (((1u << part) - 1u) << (h * part));
+      if (live == 0u) continue;
+      const unsigned char* base = reinterpret_cast<const unsigned char*>(P.replicas[i]);
+      float2 sq2 = make_float2(0.0f, 0.0f);                // two running sums (packed fp32 pairs of sm_100)
+      uint32_t rem = live;
+#pragma unroll 1
+      while (rem) {
+        const uint32_t sp0 = (uint32_t)__ffs((int)rem) - 1u;
+        uint32_t c, c_end;
+        if (whole) { c = sp0 << sh; c_end = c + (1u << sh); rem &= rem - 1u; }
+        else { c = sp0 >> sh; c_end = c + 1u; rem &= ~(((1u << (1u << sh)) - 1u) << (c << sh)); }
+#pragma unroll 1
+        for (; c < c_end; ++c) {
+          const uint32_t q = n++;
+          const uint32_t off = c * 512u + (uint32_t)lane * 16u;
+          const uint32_t el = off / kRB, sp = el >> lgP;
+          const uint32_t j_sp = __shfl_sync(0xFFFFFFFFu, j_l, (int)sp);
+          if (!((live >> sp) & 1u)) continue;              // this lane's 16 bytes are not stale ones
+          unsigned char* sc = buffer + q * 512u + (uint32_t)lane * 16u;
+          const unsigned char* old = base + rep_index(P, i, j_sp, e0 + el) * kRB;
+          if (pass == 0) {
+            if (q < G.rd_cap) cp_async16(smem_u32(sc), old);
+          } else {
+            // each lane reads back what it copied itself; a chunk the scratch had no room for comes from memory now
+            const uint4 ov = q < G.rd_cap ? *reinterpret_cast<const uint4*>(sc) : __ldcs(reinterpret_cast<const uint4*>(old));
+            const uint4 wv = *reinterpret_cast<const uint4*>(wt + off);
+            const uint32_t ow[4] = {ov.x, ov.y, ov.z, ov.w}, ww[4] = {wv.x, wv.y, wv.z, wv.w};
+            if constexpr (RT::kVecs == 2) {                // fp32 replicas: one element per word
+#pragma unroll
+              for (int h = 0; h < 4; h += 2) {
+                const float2 d = __fadd2_rn(make_float2(__uint_as_float(ow[h]), __uint_as_float(ow[h + 1])),
+                                            make_float2(-__uint_as_float(ww[h]), -__uint_as_float(ww[h + 1])));
+                sq2 = __fadd2_rn(sq2, __fmul2_rn(d, d));
+              }
+            } else {                                        // bf16 replicas: two elements per word
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const float2 d = __fadd2_rn(make_float2(__uint_as_float(ow[h] << 16), __uint_as_float(ow[h] & 0xFFFF0000u)),
+                                            make_float2(-__uint_as_float(ww[h] << 16), -__uint_as_float(ww[h] & 0xFFFF0000u)));
+                sq2 = __fadd2_rn(sq2, __fmul2_rn(d, d));
+              }
+            }
+          }
+        }
+      }
+      if (pass == 1) {
+        const float tot = warp_sum(__fadd_rn(sq2.x, sq2.y));
+        if (lane == 0) warp_acc[h * kMaxW + i] += (double)tot;   // one accumulator per replica and part, touched by one warp alone
+      }
+    }
+  };
   if (warp == CW) {
     // ================================= mask warp =================================
     uint32_t slot = 0, par = 0;
@@ -337,18 +413,48 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
       }
     }
     bulk_wait0();
+  } else if (kND > 0 && warp > CW + kNP + 1 + kNR) {
+    // ================================ drift warps ================================
+    // (wide RD builds) warp d takes replicas d, d + kND, ...: requests a tile's stale copies when its masks are
+    // published, uses them when its wire tile is, and releases both
+    const uint32_t dw = (uint32_t)(warp - CW - kNP - 2 - kNR);
+    unsigned char* scratch = rscratch + (size_t)dw * rd_buf;
+    uint32_t slot = 0, mpar = 0, wslot = 0, wpar = 0;
+    bool ok = true;
+    for (uint32_t tile = blockIdx.x; ok && tile < G.num_tiles; tile += gridDim.x) {
+      if (!mbar_wait(mfull_bar(slot), mpar, abort_flag)) break;
+      const TileMasks& tm = ring[slot];
+#pragma unroll 1
+      for (int pass = 0; pass < 2; ++pass) {
+        if (pass == 1) {
+          if (!mbar_wait(wfull_bar(wslot), wpar, abort_flag)) { ok = false; break; }
+          asm volatile("cp.async.wait_all;" ::: "memory");
+        }
+        drift_pass(tm, dw, kND, scratch, pass, wring + (size_t)wslot * kRowR);
+      }
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(wempty_bar(wslot));
+        mbar_arrive(mempty_bar(slot));
+      }
+      if (++slot == kGatherRing) { slot = 0; mpar ^= 1u; }
+      if (++wslot == kWireRing) { wslot = 0; wpar ^= 1u; }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
   } else if (warp > CW + kNP + 1) {
     // =============================== replica warps ===============================
     const uint32_t rw = (uint32_t)(warp - CW - kNP - 2);    // this warp owns replicas rw, rw + kNR, ...
-    constexpr int kChunks = kRowR / 512u;                   // a replica's row of a tile in 512-byte chunks
-    constexpr uint32_t kElemsPerChunk = 512u / kRB;
-    unsigned char* scratch = rscratch + (size_t)rw * 2u * kRdBuf;
+    constexpr bool kReadsStale = RD && kND == 0;            // twin RD: these warps also take the drift terms
+    unsigned char* scratch = rscratch + (size_t)rw * 2u * rd_buf;
     uint32_t slot = 0, wslot = 0, wpar = 0, mpar = 0, buf = 0;
-    // RD: PASS 0 requests the old copies of a tile's stale (replica, sub-packet) pairs into scratch buffer `b`
+    // twin RD: the walk of this warp's replicas' rows, unrolled over a row's few chunks (measured faster here than the
+    // drift warps' loop over the stale chunks). PASS 0 requests the old copies of a tile's stale (replica, sub-packet)
+    // pairs into scratch buffer `b`
     // (chunk after chunk in the order (replica, chunk)); pass 1 takes their squared differences against the wire
     // tile: fp32 per lane within a replica's chunks, one warp reduction per replica and tile, fp64 from there on
     // (each replica has one accumulator, touched by this warp alone, in tile order).
-    auto drift_pass = [&](const TileMasks& tm, uint32_t b, int pass, const unsigned char* wt) {
+    auto row_pass = [&](const TileMasks& tm, uint32_t b, int pass, const unsigned char* wt) {
       const uint64_t stale_l = tm.stale[lane & (kMaxSub - 1)];
       const uint32_t j_l = tm.j[lane & (kMaxSub - 1)];
       const uint32_t live_tile = (1u << tm.npk) - 1u;       // entries behind a short last tile are marked stale everywhere
@@ -369,7 +475,7 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
           const uint32_t el = off / kRB, sp = el >> lgP;
           const uint32_t j_sp = __shfl_sync(0xFFFFFFFFu, j_l, (int)sp);
           const bool mine = (live >> sp) & 1u;                                  // this lane's 16 bytes are stale ones
-          unsigned char* sc = scratch + (size_t)b * kRdBuf + q * 512u + (uint32_t)lane * 16u;
+          unsigned char* sc = scratch + (size_t)b * rd_buf + q * 512u + (uint32_t)lane * 16u;
           if (pass == 0) {
             if (mine) cp_async16(smem_u32(sc), base + rep_index(P, i, j_sp, e0 + el) * kRB);
           } else if (mine) {
@@ -399,19 +505,19 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
         }
       }
     };
-    if constexpr (RD) {
+    if constexpr (kReadsStale) {
       if (blockIdx.x < G.num_tiles) {
-        if (mbar_wait(mfull_bar(0), 0u, abort_flag)) drift_pass(ring[0], 0u, 0, nullptr);
+        if (mbar_wait(mfull_bar(0), 0u, abort_flag)) row_pass(ring[0], 0u, 0, nullptr);
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     }
     for (uint32_t tile = blockIdx.x; tile < G.num_tiles; tile += gridDim.x) {
-      if constexpr (RD) {
+      if constexpr (kReadsStale) {
         // the next tile's old copies first: they have this tile's duration to arrive
         if (tile + gridDim.x < G.num_tiles) {
           const uint32_t nslot = slot + 1u == kGatherRing ? 0u : slot + 1u;
           if (!mbar_wait(mfull_bar(nslot), nslot == 0u ? mpar ^ 1u : mpar, abort_flag)) break;
-          drift_pass(ring[nslot], buf ^ 1u, 0, nullptr);
+          row_pass(ring[nslot], buf ^ 1u, 0, nullptr);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
       }
@@ -440,9 +546,9 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
                    *reinterpret_cast<const uint4*>(wt + off));
         }
       }
-      if constexpr (RD) {
+      if constexpr (kReadsStale) {
         asm volatile("cp.async.wait_group 1;" ::: "memory");   // everything but the next tile's requests has landed
-        drift_pass(tm, buf, 1, wt);
+        row_pass(tm, buf, 1, wt);
         buf ^= 1u;
       }
       __syncwarp();
@@ -453,7 +559,7 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
       if (++slot == kGatherRing) { slot = 0; mpar ^= 1u; }
       if (++wslot == kWireRing) { wslot = 0; wpar ^= 1u; }
     }
-    if constexpr (RD) asm volatile("cp.async.wait_all;" ::: "memory");
+    if constexpr (kReadsStale) asm volatile("cp.async.wait_all;" ::: "memory");
   } else {
     // =============================== compute warps ===============================
     const uint32_t idx = threadIdx.x * kEpl;               // first element of this lane within the tile
@@ -607,7 +713,7 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
     if (threadIdx.x < kMaxW) {
       double t = 0.0;
 #pragma unroll
-      for (int w = 0; w < CW; ++w) t += warp_acc[w * kMaxW + threadIdx.x];
+      for (int w = 0; w < kAccRows; ++w) t += warp_acc[w * kMaxW + threadIdx.x];
       P.partials[(size_t)blockIdx.x * kMaxW + threadIdx.x] = t;
     }
     if (P.ticket) drift_last_block(P, warp, lane, GatherShape<CW, RD>::kThreads / 32);

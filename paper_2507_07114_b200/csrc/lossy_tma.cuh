@@ -62,6 +62,8 @@ struct TmaGeom {
   uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores, bit 2 (gather pipeline): L2 prefetch of stale copies
   uint32_t packets_per_tile;  // PACKED build: whole small packets per tile (2, 4 or 8), else 1
   uint32_t full_packets;      // PACKED build: complete packets of the bucket
+  uint32_t rd_cap;            // gather pipeline, RD builds: 512-byte chunks per scratch buffer
+  uint32_t rd_lgsplit;        // gather pipeline, wide RD builds: log2 of the parts a replica's row of a tile is cut into
   uint32_t* status;           // device status word (0 = fine)
 };
 

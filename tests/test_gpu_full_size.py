@@ -26,8 +26,8 @@ def _slabs(w, rng, n_random, width):
     return sorted(starts)
 
 
-def _run_full(w, steps, slab_packets, n_random, full_drift):
-    gpu = GpuRun(w)
+def _run_full(w, steps, slab_packets, n_random, full_drift, flags=0):
+    gpu = GpuRun(w, flags=flags)
     rng = np.random.default_rng(0)
     slabs = _slabs(w, rng, n_random, slab_packets)
     P = w.packet_elems
@@ -113,21 +113,30 @@ def test_w64_high_loss_full_size_split_build_with_staged_stale_copies():
 
 
 def test_config5_point_full_size_small_packets_register_path():
-    # P=256 takes the register-path kernel at full size
+    # the register-path kernel at full size (what P = 256 ran on at high loss before the drift-warp build; still the
+    # kernel of many workers at high loss)
     w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.3)
-    _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False)
+    gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=False, flags=L.LOSSY_REGISTER_PATH)
+    assert L.lossy_describe_plan(gpu.ctx) == "register kernel"
+
+
+def test_config5_point_full_size_small_packets_high_loss_drift_warps():
+    # P = 256, p = 0.3: the wide gather build whose drift warps read the stale copies
+    w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.3)
+    gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=True)
+    assert L.lossy_describe_plan(gpu.ctx) == "gather wide packets/tile=8 stages=3 drift-warps"
 
 
 def test_config5_point_full_size_small_packets_gather_pipeline():
     # P=256 at low and moderate loss takes the gather pipeline (eight whole packets per tile) at full size
     w = workload.scaled(CFG["cfg5_w16_layer_sweep"], workload.LAYER_ELEMS, packet_elems=256, p=0.1)
     gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=True)
-    assert L.lossy_describe_plan(gpu.ctx) == "gather wide packets/tile=8 stages=3"
+    assert L.lossy_describe_plan(gpu.ctx) == "gather wide packets/tile=8 stages=3 drift-warps"
 
 
 def test_few_workers_small_packets_full_size_gather_twin():
-    # W = 4, P = 256 at high loss: the twin gather build whose replica warps also read the stale copies
-    w = workload.scaled(CFG["cfg2_w8_layer_adam"], workload.LAYER_ELEMS, W=4, packet_elems=256, p=0.3)
+    # W = 3, P = 256 at high loss: the twin gather build whose replica warps also read the stale copies
+    w = workload.scaled(CFG["cfg2_w8_layer_adam"], workload.LAYER_ELEMS, W=3, packet_elems=256, p=0.3)
     gpu = _run_full(w, steps=2, slab_packets=24, n_random=4, full_drift=True)
     assert L.lossy_describe_plan(gpu.ctx) == "gather twin packets/tile=4 stages=4"
 

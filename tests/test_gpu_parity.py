@@ -106,6 +106,14 @@ EDGE = [
     # the gather pipeline where the policy would pick the register kernel: many stale copies per sub-packet
     ("gather_forced_w24_high_loss", 24, 256 * 70 + 8, 256, 0.4, "adam", "bf16", "bf16", L.LOSSY_GATHER_PATH),
     ("gather_forced_w64_f32_replicas", 64, 512 * 33, 512, 0.3, "sgd", "bf16", "f32", L.LOSSY_GATHER_PATH),
+    # the wide gather build with drift warps: replica rows cut into halves (W = 12) and quarters (W = 5, W = 4), whole
+    # rows with more stale chunks than the scratch holds (W = 24), fp32 replicas (sixteen chunks per row)
+    ("packed_drift_warps_w12_halves", 12, 256 * 67 + 9, 256, 0.3, "adam", "bf16", "bf16", 0),
+    ("packed_drift_warps_w5_quarters_512", 5, 512 * 41, 512, 0.2, "sgd", "f32", "bf16", 0),
+    ("packed_drift_warps_w24_scratch_overflow", 24, 256 * 130 + 8, 256, 0.3, "adam", "bf16", "bf16", 0),
+    ("packed_drift_warps_w7_f32_replicas", 7, 256 * 90, 256, 0.45, "adam", "bf16", "f32", 0),
+    ("packed_drift_warps_w4_wide", 4, 256 * 75 + 100, 256, 0.3, "adam", "bf16", "bf16", SKIP),
+    ("packed_drift_warps_w17_elided", 17, 512 * 40, 512, 0.25, "sgd", "bf16", "bf16", L.LOSSY_REPLICA_SKIP_OWNER),
 ]
 
 
@@ -329,11 +337,16 @@ def test_launch_policy_picks_the_expected_build_for_the_benchmark_configurations
     assert plan(64, 4096, 0.1)[0] == "bulk-copy twin group=8 stale=late stages=3"         # config 3
     assert plan(4, 1024, 0.1, gd="f32", rd="f32")[0].startswith("bulk-copy twin group=4")  # config 1
     assert plan(16, 1024, 0.3)[0] == "bulk-copy twin group=8 stale=early stages=3"        # config 5, P = 1024
-    assert plan(16, 256, 0.1)[0] == "gather wide packets/tile=8 stages=3"                  # config 5, small packets, low loss
+    assert plan(16, 256, 0.1)[0] == "gather wide packets/tile=8 stages=3 drift-warps"      # config 5, small packets
     assert plan(16, 1024, 0.05)[0].startswith("bulk-copy wide group=8 stale=late packed")  # config 5, P = 1024, low loss: two packets per wide tile
-    assert plan(16, 256, 0.3)[0] == "register kernel"                                     # ... and at high loss with many workers
-    assert plan(8, 256, 0.3)[0] == "gather wide packets/tile=8 stages=3"
-    assert plan(4, 256, 0.3)[0] == "gather twin packets/tile=4 stages=4"                  # few workers: twin geometry
+    assert plan(16, 256, 0.3)[0] == "gather wide packets/tile=8 stages=3 drift-warps"      # ... at high loss too
+    assert plan(16, 256, 0.1)[1] == "gather wide packets/tile=8 stages=3"                  # no drift norms asked for
+    assert plan(17, 256, 0.5)[0] == "register kernel"                                     # eight stale replicas per sub-packet
+    assert plan(32, 256, 0.05)[0] == "gather wide packets/tile=8 stages=3"                 # many workers: the compute warps read the stale copies
+    assert plan(32, 256, 0.2)[0] == "register kernel"
+    assert plan(8, 256, 0.3)[0] == "gather wide packets/tile=8 stages=3 drift-warps"
+    assert plan(4, 256, 0.3)[0] == "gather wide packets/tile=8 stages=4 drift-warps"
+    assert plan(3, 256, 0.3)[0] == "gather twin packets/tile=4 stages=4"                  # two or three workers: twin geometry
     assert plan(40, 128, 0.1)[0].startswith("gather twin packets/tile=8")                 # 128 elements: only the twin tile packs them
     assert plan(16, 256, 0.1, flags=L.LOSSY_PACKED_BULK)[0].startswith("bulk-copy wide group=8 stale=late packed")
     assert plan(64, 4096, 0.3)[0] == "bulk-copy twin group=8 stale=staged split stages=4"
