@@ -407,21 +407,26 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
   const TmaPolicy t = tma_policy(ctx->cfg);
   if (!(ctx->cfg.flags & LOSSY_PACKED_BULK) && ctx->cfg.packet_elems < (uint32_t)TmaShape<8>::kTile) {
     // Packets shorter than a tile (128, 256 or 512 elements): the gather pipeline, where it beats the register
-    // kernel (fractions of the copy rate, 20 steps of a 202 M element bucket).
-    //  * 4..24 workers, packets of 256 or 512 elements, fewer than 7.5 stale replicas per sub-packet: the wide
-    //    geometry with drift warps of its own (W = 16, P = 256: 1.00 / 0.96 / 0.94 / 0.90 / 0.85 at p = 0 / 0.05 /
-    //    0.1 / 0.2 / 0.3, where the compute warps' reads gave 0.94 / 0.94 / 0.96 / 0.81 / 0.70 and the register
-    //    kernel 0.91 / 0.84 / 0.82 / 0.79 / 0.76; W = 8: 0.97 and 0.84 at p = 0.1 and 0.3 against 0.91 and 0.78;
-    //    W = 24, p = 0.3: 0.81 against 0.72; W = 4: 0.80-0.83 against 0.75-0.81 for the twin geometry);
-    //  * beyond that the drift warps fall behind (W = 17, p = 0.5: 0.43): many workers at high loss stay with the
-    //    register kernel (p = 0.3, W >= 12: 0.71-0.77 against 0.65-0.77; p = 0.2, W = 32: 0.85 against 0.79-0.84),
-    //    the rest with the compute warps' reads (W = 32, p = 0.05: 0.96 against 0.91; W = 64, p = 0.1: 0.89);
+    // kernel. Fractions of the copy rate, 20 steps of a 202 M element bucket, P = 256, taken back to back in one
+    // process (power-capped clocks; a point measured alone runs 3-6 % higher), S = (W - 1) p_param = stale replicas
+    // per sub-packet:
+    //  * the wide geometry with drift warps of its own for 4..24 workers, packets of 256 or 512 elements and
+    //    0.2 (W - 8) <= S < 7.5 (W = 8: 0.97 / 0.97 / 0.94 / 0.85 at p = 0.05 / 0.1 / 0.2 / 0.3, where the compute
+    //    warps' reads gave 0.89 / 0.84 / 0.82 / 0.77 and the register kernel 0.77 and 0.67 at p = 0.1 and 0.3; W = 16:
+    //    0.92 / 0.88 / 0.84 at p = 0.1 / 0.2 / 0.3 against 0.90 / 0.81 / 0.69, register kernel 0.82 / 0.79 / 0.76;
+    //    W = 24: 0.83 and 0.78 at p = 0.2 and 0.3 against 0.81 and 0.72; W = 4: 0.77-0.83 against 0.75-0.84 for the
+    //    twin geometry);
+    //  * below that band (many workers, few stale copies) the compute warps' reads stay ahead (W = 16, p = 0.05: 0.98
+    //    against 0.91; W = 24, p = 0.1: 0.88 against 0.85; W = 32, p = 0.05: 0.96 against 0.91);
+    //  * above it the drift warps fall behind (W = 17, p = 0.5: 0.43): many workers at high loss stay with the
+    //    register kernel (p = 0.2, W = 32: 0.85 against 0.79-0.84; W = 17, p = 0.5: 0.56);
     //  * two or three workers, and packets of 128 elements: the twin geometry (W = 2: 0.78-0.81 against 0.69-0.74
     //    for the wide one), whose replica warps also read the stale copies up to four workers.
     const lossy_config& c = ctx->cfg;
     const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
     const bool wide_fits = c.packet_elems * (uint32_t)kMaxSub >= (uint32_t)GatherShape<16>::kTile;
-    const bool drift_warps = wide_fits && c.W >= 4u && c.W <= 24u && (c.W - 1u) * c.p_param < 7.5;
+    const double stale = (c.W - 1u) * c.p_param;
+    const bool drift_warps = wide_fits && c.W >= 4u && c.W <= 24u && stale < 7.5 && stale >= 0.2 * ((double)c.W - 8.0);
     const bool reg_ahead = !(c.flags & LOSSY_GATHER_PATH) && !drift_warps && ((c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15));
     if (!reg_ahead) {
       int rc = LOSSY_OK;

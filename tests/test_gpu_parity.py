@@ -337,10 +337,10 @@ def test_launch_policy_picks_the_expected_build_for_the_benchmark_configurations
     assert plan(64, 4096, 0.1)[0] == "bulk-copy twin group=8 stale=late stages=3"         # config 3
     assert plan(4, 1024, 0.1, gd="f32", rd="f32")[0].startswith("bulk-copy twin group=4")  # config 1
     assert plan(16, 1024, 0.3)[0] == "bulk-copy twin group=8 stale=early stages=3"        # config 5, P = 1024
-    assert plan(16, 256, 0.1)[0] == "gather wide packets/tile=8 stages=3 drift-warps"      # config 5, small packets
+    assert plan(16, 256, 0.1)[0] == "gather wide packets/tile=8 stages=3"                  # config 5, small packets, low loss
     assert plan(16, 1024, 0.05)[0].startswith("bulk-copy wide group=8 stale=late packed")  # config 5, P = 1024, low loss: two packets per wide tile
-    assert plan(16, 256, 0.3)[0] == "gather wide packets/tile=8 stages=3 drift-warps"      # ... at high loss too
-    assert plan(16, 256, 0.1)[1] == "gather wide packets/tile=8 stages=3"                  # no drift norms asked for
+    assert plan(16, 256, 0.3)[0] == "gather wide packets/tile=8 stages=3 drift-warps"      # ... at high loss: drift warps
+    assert plan(16, 256, 0.3)[1] == "gather wide packets/tile=8 stages=3"                  # no drift norms asked for
     assert plan(17, 256, 0.5)[0] == "register kernel"                                     # eight stale replicas per sub-packet
     assert plan(32, 256, 0.05)[0] == "gather wide packets/tile=8 stages=3"                 # many workers: the compute warps read the stale copies
     assert plan(32, 256, 0.2)[0] == "register kernel"
