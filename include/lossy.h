@@ -54,7 +54,8 @@ extern "C" {
 typedef struct lossy_ctx lossy_ctx; /* opaque; host object + small device scratch */
 
 enum { LOSSY_OK = 0, LOSSY_EINVAL = 1, LOSSY_ENOMEM = 2, LOSSY_ECUDA = 3, LOSSY_EDEVICE = 4,
-       LOSSY_ELIMIT = 5 /* a size is beyond what drift_norms_static supports */ };
+       LOSSY_ELIMIT = 5 /* a size is beyond what drift_norms_static supports */,
+       LOSSY_EDEVCHECK = 6 /* debug build only: a kernel's index check failed (lossy_device_status) */ };
 enum { LOSSY_F32 = 0, LOSSY_BF16 = 1 };  /* element types of gradients / replicas */
 enum { LOSSY_SGD = 0, LOSSY_ADAM = 1 };
 enum {
@@ -387,6 +388,33 @@ int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* targ
  * lossy_reset_status clears it.
  */
 int lossy_device_status(lossy_ctx* ctx, void* stream);
+
+/*
+ * Debug build. The same sources compiled with -DLOSSY_DEVCHECK give a second
+ * library (liblossy_b200_check.so) with the same entry points, in which every
+ * kernel of the step path (register kernel, fused and single-phase bulk-copy
+ * pipelines, gather pipeline) checks, before it touches memory for a chunk or
+ * tile, that the packet index is one of the context's packets, that the element
+ * range lies inside the slab, and that every replica's range (through the
+ * owner-elided index map where that layout is on) lies inside that replica's
+ * array. A range that fails is recorded (first failure wins: kernel, array kind,
+ * offset, length) and is not touched: the register kernel skips the chunk, a
+ * pipeline stops through its bounded-wait exit. Nothing traps or asserts. The
+ * next lossy_device_status returns LOSSY_EDEVCHECK with the record in
+ * lossy_last_error; lossy_reset_status clears it. The checks stand in for a
+ * memory-checking tool where none can be run; the normal build contains none of
+ * them (they compile to nothing) and never returns LOSSY_EDEVCHECK.
+ *
+ * lossy_has_device_checks — 1 in the debug build, 0 in the normal one.
+ *
+ * lossy_selftest_shrink_checks — a test hook of the debug build: from the next
+ * call on, the checks hold every range against n - elems elements instead of n
+ * (elems = 0 restores n), so that ranges near the end fail their check although
+ * the arrays behind them are whole: the failure report runs without an access
+ * out of bounds. LOSSY_EINVAL in the normal build. The paper has no counterpart.
+ */
+int lossy_has_device_checks(void);
+int lossy_selftest_shrink_checks(lossy_ctx* ctx, uint64_t elems);
 
 /*
  * lossy_reset_status — clear the context's device status word and its

@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE, LOSSY_ELIMIT = 0, 1, 2, 3, 4, 5
+LOSSY_OK, LOSSY_EINVAL, LOSSY_ENOMEM, LOSSY_ECUDA, LOSSY_EDEVICE, LOSSY_ELIMIT, LOSSY_EDEVCHECK = 0, 1, 2, 3, 4, 5, 6
 LOSSY_F32, LOSSY_BF16 = 0, 1
 LOSSY_SGD, LOSSY_ADAM = 0, 1
 LOSSY_SELF_LOSSLESS, LOSSY_ZERO_SKIP, LOSSY_REGISTER_PATH, LOSSY_REPLICA_SKIP_OWNER, LOSSY_PACKED_BULK = 1, 2, 4, 8, 16
@@ -25,6 +25,7 @@ EXPORTS = [
     "drift_norms", "drift_pairwise", "drift_norms_static", "lossy_fused_step", "lossy_aggregate_alg1", "lossy_fused_step_alg1", "lossy_fused_step_host", "lossy_mask", "lossy_hash_u32",
     "lossy_mask_grid", "lossy_closed_loop_grads", "lossy_device_status", "lossy_last_error", "lossy_num_packets", "lossy_kernel_launches",
     "lossy_describe_plan", "lossy_replica_elems", "lossy_reset_status", "lossy_selftest_wait_expiry",
+    "lossy_has_device_checks", "lossy_selftest_shrink_checks",
 ]
 
 
@@ -47,12 +48,19 @@ class LossyError(RuntimeError):
 _lib = None
 
 
+def default_library_path() -> str:
+    """The library this process binds to: the debug build (index checks in every kernel of the step path) when the
+    environment says LOSSY_B200_CHECKED=1, else the normal one. Read once, at the first call."""
+    return _build.CHECK_LIB_PATH if os.environ.get("LOSSY_B200_CHECKED") == "1" else _build.LIB_PATH
+
+
 def load_library(path: str | None = None) -> C.CDLL:
     """dlopen liblossy_b200.so (built in-tree by paper_2507_07114_b200.build) and declare its signatures."""
     global _lib
     if _lib is not None and path is None:
         return _lib
-    path = path or _build.LIB_PATH
+    default = default_library_path()
+    path = path or default
     if not os.path.exists(path):
         raise FileNotFoundError(f"{path} is missing: run paper_2507_07114_b200.build.build() (needs nvcc); "
                                 "there is no CPU fallback")
@@ -112,9 +120,13 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.lossy_reset_status.argtypes = [vp, vp]
     lib.lossy_selftest_wait_expiry.restype = C.c_int
     lib.lossy_selftest_wait_expiry.argtypes = [vp, u32, vp]
+    lib.lossy_has_device_checks.restype = C.c_int
+    lib.lossy_has_device_checks.argtypes = []
+    lib.lossy_selftest_shrink_checks.restype = C.c_int
+    lib.lossy_selftest_shrink_checks.argtypes = [vp, u64]
     lib.lossy_describe_plan.restype = C.c_int
     lib.lossy_describe_plan.argtypes = [vp, C.c_int, C.c_char_p, C.c_size_t]
-    if path == _build.LIB_PATH:
+    if path == default:
         _lib = lib
     return lib
 
@@ -276,6 +288,14 @@ def lossy_reset_status(ctx):
 
 def lossy_selftest_wait_expiry(ctx, max_polls: int = 1024):
     _check(ctx, load_library().lossy_selftest_wait_expiry(ctx, max_polls, _stream()))
+
+
+def lossy_has_device_checks() -> bool:
+    return bool(load_library().lossy_has_device_checks())
+
+
+def lossy_selftest_shrink_checks(ctx, elems: int):
+    _check(ctx, load_library().lossy_selftest_shrink_checks(ctx, elems))
 
 
 def lossy_replica_elems(ctx, worker: int) -> int:

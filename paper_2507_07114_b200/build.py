@@ -8,6 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "liblossy_b200.so")
+CHECK_LIB_PATH = os.path.join(PKG_DIR, "liblossy_b200_check.so")   # the debug build: -DLOSSY_DEVCHECK (index checks in the kernels)
 SOURCES = ["lossy_api.cu", "lossy_noalloc.cu"]
 HEADERS = ["lossy_device.cuh", "lossy_kernels.cuh", "lossy_tma.cuh", "lossy_gather.cuh", "lossy_phase_tma.cuh", os.path.join("..", "..", "include", "lossy.h")]
 
@@ -18,27 +19,36 @@ NVCC_FLAGS = [
 ]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def _stale(lib: str) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, s) for s in SOURCES + HEADERS] + [os.path.abspath(__file__)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile liblossy_b200.so next to this file; returns its path."""
-    if not force and not _stale():
-        return LIB_PATH
+    """Compile liblossy_b200.so and its debug twin liblossy_b200_check.so next to this file (the two nvcc runs side by
+    side); returns the path of the normal library."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", LIB_PATH + ".tmp",
-           *[os.path.join(CSRC, s) for s in SOURCES]]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose:
-        sys.stderr.write(res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    os.replace(LIB_PATH + ".tmp", LIB_PATH)
+    jobs = []
+    for lib, extra in ((LIB_PATH, []), (CHECK_LIB_PATH, ["-DLOSSY_DEVCHECK=1"])):
+        if not force and not _stale(lib):
+            continue
+        cmd = [nvcc, *NVCC_FLAGS, *extra, *(["-Xptxas", "-v"] if verbose and not extra else []), "-o", lib + ".tmp",
+               *[os.path.join(CSRC, s) for s in SOURCES]]
+        jobs.append((lib, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True)))
+    failed = []
+    for lib, proc in jobs:
+        out, err = proc.communicate()
+        if verbose:
+            sys.stderr.write(err)
+        if proc.returncode != 0:
+            failed.append(os.path.basename(lib) + ":\n" + out + err)
+        else:
+            os.replace(lib + ".tmp", lib)
+    if failed:
+        raise RuntimeError("nvcc failed:\n" + "\n".join(failed))
     return LIB_PATH
 
 

@@ -25,7 +25,8 @@ struct lossy_ctx {
   int num_sms;
   uint32_t max_blocks;   // capacity of `partials`
   double* partials;      // device, [max_blocks][kMaxW], followed by the status word
-  uint32_t* status;      // device status word: 0 = fine, 1 = a bounded wait in a kernel gave up
+  uint32_t* status;      // device status words: [0] 0 = fine, 1 = a bounded wait in a kernel gave up; [1..4] debug build: a failed index check
+  uint64_t check_shrink; // debug build self-test: the index checks hold ranges against n - check_shrink
   uint32_t* ticket;      // device counter of finished blocks (last-block drift finalisation), zero between calls
   bool plan_only;        // launch helpers only report their grid size
   const uint64_t* reliable;  // caller-owned device array [2][K] of reliable-link bits, or NULL
@@ -110,6 +111,8 @@ void fill_common(const lossy_ctx* ctx, uint64_t step, Params& P) {
   P.partials = ctx->partials;
   P.K = (uint32_t)ctx->K;
   P.reliable = ctx->reliable;
+  P.check = ctx->status + 1;
+  P.check_n = c.n - (ctx->check_shrink < c.n ? ctx->check_shrink : c.n);
   fill_rep_skip(P, (c.flags & LOSSY_REPLICA_SKIP_OWNER) != 0);
   if (ctx->burst_state) {
     // the states after step t-1 live in buffer (t-1)&1, those after step t go to buffer t&1
@@ -1031,17 +1034,35 @@ int lossy_closed_loop_grads(lossy_ctx* ctx, const float* curv, const float* targ
 
 int lossy_device_status(lossy_ctx* ctx, void* stream) {
   if (!ctx) return LOSSY_EINVAL;
-  uint32_t word = 0;
-  cudaError_t e = cudaMemcpyAsync(&word, ctx->status, sizeof word, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+  uint32_t word[5] = {0, 0, 0, 0, 0};
+  cudaError_t e = cudaMemcpyAsync(word, ctx->status, sizeof word, cudaMemcpyDeviceToHost, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(ctx, "status read", e);
-  if (word != 0) return fail(ctx, LOSSY_EDEVICE, "a bounded wait inside a kernel gave up; results of that call are invalid");
+  if (word[1] != 0) {   // debug build only; a pipeline that skipped a tile also left through its wait exit (word[0])
+    static const char* const kSites[] = {"?", "register kernel", "fused bulk-copy pipeline (packed)", "fused bulk-copy pipeline",
+                                         "single-phase bulk-copy pipeline", "gather pipeline"};
+    const uint32_t site = word[1] & 15u;
+    snprintf(ctx->err, sizeof ctx->err, "device index check failed in the %s: %s elements [%llu, +%u) lie outside the array; not touched, the results of that call are invalid",
+             site < 6 ? kSites[site] : kSites[0], (word[1] & kSiteReplica) ? "replica" : "slab",
+             (unsigned long long)(((uint64_t)word[3] << 32) | word[2]), word[4]);
+    return LOSSY_EDEVCHECK;
+  }
+  if (word[0] != 0) return fail(ctx, LOSSY_EDEVICE, "a bounded wait inside a kernel gave up; results of that call are invalid");
+  return LOSSY_OK;
+}
+
+int lossy_has_device_checks(void) { return kDevCheck ? 1 : 0; }
+
+int lossy_selftest_shrink_checks(lossy_ctx* ctx, uint64_t elems) {
+  if (!ctx) return LOSSY_EINVAL;
+  if (!kDevCheck) return fail(ctx, LOSSY_EINVAL, "this library was built without device index checks");
+  ctx->check_shrink = elems;
   return LOSSY_OK;
 }
 
 int lossy_reset_status(lossy_ctx* ctx, void* stream) {
   if (!ctx) return LOSSY_EINVAL;
-  cudaError_t e = cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), (cudaStream_t)stream);
+  cudaError_t e = cudaMemsetAsync(ctx->status, 0, 5 * sizeof(uint32_t), (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->ticket, 0, sizeof(uint32_t), (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(ctx, "status reset", e);
   ctx->err[0] = 0;

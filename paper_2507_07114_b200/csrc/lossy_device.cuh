@@ -70,6 +70,11 @@ struct Params {
   // Owner-elided replicas (kSkipOwner): replica i stores this context's elements WITHOUT the packets worker i
   // owns, so everything behind worker i's shard sits rep_skip[i] elements lower in its array. All zero otherwise.
   uint64_t rep_skip[kMaxW];
+  // Debug build (LOSSY_DEVCHECK): where a failed index check is recorded (4 words: site, element offset low and
+  // high, length; the first failure wins) and the element count the checks hold a range against (n, or less when
+  // the self-test shrinks it). Unused otherwise.
+  uint32_t* check;
+  uint64_t check_n;
 };
 
 // Owner-elided replicas: rep_skip[i] = elements of worker i's shard inside the context's packet range
@@ -91,6 +96,51 @@ __host__ inline void fill_rep_skip(Params& P, bool elide) {
 __device__ __forceinline__ uint64_t rep_index(const Params& P, uint32_t i, uint32_t j, uint64_t e) {
   return e - (j > i ? P.rep_skip[i] : 0ull);
 }
+// Debug build (compiled with -DLOSSY_DEVCHECK, a library of its own): before a kernel of the step path touches
+// memory for a chunk or tile it checks the element range and the packet index against the context's sizes, and
+// every replica's range (through the owner-elided index map) against that replica's length. A range that fails
+// is recorded in Params::check and not touched: the register kernel skips the chunk, a pipeline raises its abort
+// flag and every role leaves through the bounded-wait exit. Nothing traps or asserts. In the normal build all of
+// this compiles to nothing.
+#ifdef LOSSY_DEVCHECK
+constexpr bool kDevCheck = true;
+#else
+constexpr bool kDevCheck = false;
+#endif
+enum CheckSite : uint32_t { kSiteRegister = 1, kSiteFusedPacked = 2, kSiteFused = 3, kSitePhase = 4, kSiteGather = 5, kSiteReplica = 16 };
+__device__ __forceinline__ void check_record(const Params& P, uint32_t site, uint64_t e0, uint64_t len) {
+  if (atomicCAS(&P.check[0], 0u, site) == 0u) {
+    P.check[1] = (uint32_t)e0;
+    P.check[2] = (uint32_t)(e0 >> 32);
+    P.check[3] = (uint32_t)len;
+  }
+}
+// elements [e0, e0 + len) of packet k: inside the slab, and k a packet of it
+__device__ __forceinline__ bool span_ok(const Params& P, uint32_t k, uint64_t e0, uint64_t len, uint32_t site) {
+  if constexpr (!kDevCheck) return true;
+  if (!P.check) return true;      // a caller without a context (the no-allocation entry point) has nowhere to record
+  if (k < P.K && (len == 0 || (len <= P.check_n && e0 <= P.check_n - len))) return true;   // an empty range touches nothing
+  check_record(P, site, e0, len);
+  return false;
+}
+// the same elements inside replica i's array (owner j; the owner has no copy when the replicas are owner-elided)
+__device__ __forceinline__ bool rep_span_ok(const Params& P, uint32_t i, uint32_t j, uint64_t e0, uint64_t len, uint32_t site) {
+  if constexpr (!kDevCheck) return true;
+  if (!P.check || len == 0 || ((P.flags & kSkipOwner) && i == j)) return true;
+  const uint64_t limit = P.check_n - (P.rep_skip[i] < P.check_n ? P.rep_skip[i] : P.check_n);
+  const uint64_t at = e0 - (j > i ? P.rep_skip[i] : 0ull);
+  if (at <= e0 && len <= limit && at <= limit - len) return true;
+  check_record(P, site | kSiteReplica, at, len);
+  return false;
+}
+// every replica's range of a tile or chunk, the workers dealt over the lanes; warp-uniform result
+__device__ __forceinline__ bool tile_ok(const Params& P, uint32_t k, uint32_t j, uint64_t e0, uint64_t len, uint32_t site, int lane) {
+  if constexpr (!kDevCheck) return true;
+  bool ok = span_ok(P, k, e0, len, site);
+  for (uint32_t i = (uint32_t)lane; i < P.W; i += 32u) ok = rep_span_ok(P, i, j, e0, len, site) && ok;
+  return __all_sync(0xFFFFFFFFu, ok);
+}
+
 // The replica that does not exist for a packet of owner j (as a bit), or 0 with full replicas.
 __device__ __forceinline__ uint64_t own_bit(const Params& P, uint32_t j) {
   return (P.flags & kSkipOwner) ? 1ull << j : 0ull;

@@ -276,6 +276,12 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
       if (!mbar_wait(mempty_bar(slot), par ^ 1u, abort_flag)) break;
       const uint32_t kfirst = tile * G.packets_per_tile;
       const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
+      if constexpr (kDevCheck) {   // debug build: every sub-packet's range, in the slab and in every replica
+        bool fine = true;
+        for (uint32_t sp = 0; sp < npk; ++sp)
+          fine = tile_ok(P, kfirst + sp, (P.k0 + kfirst + sp) / P.pps, (uint64_t)(kfirst + sp) * P.P, P.P, kSiteGather, lane) && fine;
+        if (!fine) { *abort_flag = 1u; break; }
+      }
       TileMasks& tm = ring[slot];
       auto report = [&](uint32_t sp, uint32_t j, uint64_t r, uint64_t st, uint64_t gbad, uint64_t pbad) {   // one lane
         const uint32_t k = kfirst + sp;

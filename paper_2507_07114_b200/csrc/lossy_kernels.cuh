@@ -212,6 +212,11 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
     const uint64_t e = (uint64_t)k * P.P + in_pkt;
     int nvalid = 0;
     if (in_pkt < P.P && e < P.n) nvalid = (P.n - e >= 8) ? 8 : (int)(P.n - e);
+    if constexpr (kDevCheck) {   // debug build: the chunk's range, in the slab and in every replica
+      const uint64_t c0 = (uint64_t)k * P.P + (uint64_t)c * kChunk;
+      const uint64_t cl = c0 < P.n ? (P.n - c0 < (uint64_t)kChunk ? P.n - c0 : (uint64_t)kChunk) : 0;
+      if (!tile_ok(P, k, j, c0, cl, kSiteRegister, lane)) continue;
+    }
 
     // ---- delivery indicators of this packet (warp-uniform) -------------------
     uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;

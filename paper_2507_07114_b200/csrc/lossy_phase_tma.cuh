@@ -112,6 +112,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint32_t j = __shfl_sync(0xFFFFFFFFu, j_l, src);
         const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
         const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
+        if (!tile_ok(P, k, j, e0, len, kSitePhase, lane)) { *abort_flag = 1u; ok = false; break; }   // debug build only
         uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
         uint32_t cnt = 1;
         if constexpr (kMasked) {

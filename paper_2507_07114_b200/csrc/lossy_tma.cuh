@@ -324,6 +324,12 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
         const uint32_t npk = min(G.packets_per_tile, G.full_packets - kfirst);
         const uint64_t e0 = (uint64_t)kfirst * P.P;
         const uint32_t len = npk * P.P;
+        if constexpr (kDevCheck) {   // debug build: every sub-packet's range, in the slab and in every replica
+          bool fine = true;
+          for (uint32_t sp = 0; sp < npk; ++sp)
+            fine = tile_ok(P, kfirst + sp, (P.k0 + kfirst + sp) / P.pps, e0 + (uint64_t)sp * P.P, P.P, kSiteFusedPacked, lane) && fine;
+          if (!fine) { *abort_flag = 1u; ok = false; break; }
+        }
         for (uint32_t g = 0; g < G.groups; ++g) {
           if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag)) { ok = false; break; }
           const bool last = g + 1 == G.groups;
@@ -379,6 +385,7 @@ __global__ void __launch_bounds__(TmaShape<CW>::kThreads, TmaShape<CW>::kCtasPer
           const uint32_t j = __shfl_sync(0xFFFFFFFFu, j_l, src);
           const uint64_t e0 = (uint64_t)k * P.P + (uint64_t)c * kTile;
           const uint32_t len = min((uint32_t)kTile, P.P - c * kTile);
+          if (!tile_ok(P, k, j, e0, len, kSiteFused, lane)) { *abort_flag = 1u; ok = false; break; }   // debug build only
           uint64_t recv = 0, stale = 0, gbad = 0, pbad = 0;
           if (B > 1) batch_masks<AGG | BCAST>(P, draws, k, src, wmask, recv, stale, gbad, pbad);
           else packet_masks<AGG | BCAST>(P, k, j, lane, recv, stale, gbad, pbad);

@@ -28,6 +28,11 @@ def test_header_symbols_are_exported_and_bound():
         assert n in L.EXPORTS, f"{n} has no Python binding of the same name"
         assert callable(getattr(L, n))
     assert sorted(L.EXPORTS) == names
+    # the debug twin (-DLOSSY_DEVCHECK: index checks in the kernels) has the same entry points and says what it is
+    chk = ctypes.CDLL(B.CHECK_LIB_PATH)
+    for n in names:
+        assert hasattr(chk, n), f"{n} missing from the debug build"
+    assert lib.lossy_has_device_checks() == 0 and chk.lossy_has_device_checks() == 1
 
 
 def test_config_struct_layout_matches_the_header():
