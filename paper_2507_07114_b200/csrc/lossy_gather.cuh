@@ -16,9 +16,10 @@
 //                  in place in shared memory, and write the wire tile into a ring of its own
 //   store warp     theta / m / v back with three bulk copies; releases the stage
 //   replica warps  each owns a fixed share of the replicas: from the wire ring it stores every (replica,
-//                  sub-packet) pair that takes the broadcast, and (drift norms) loads the old copy of every pair
-//                  that misses it and accumulates the squared difference — decoupled from the tile pipeline, so
-//                  no compute warp ever waits on a global load
+//                  sub-packet) pair that takes the broadcast
+//   drift norms    the old copy of every pair that misses the broadcast is read and its squared difference from
+//                  the wire tile summed, by whichever of three the host picked: eight drift warps of their own
+//                  (wide geometry, RD), the replica warps (twin geometry, RD), or the compute warps
 // A compute warp's 128 elements lie inside one sub-packet (packets here are powers of two from 128 elements
 // that divide the tile). Every wait is bounded as in the other pipelines. No cluster, no multicast.
 #pragma once
