@@ -214,7 +214,8 @@ __global__ void __launch_bounds__(kThreads, LOSSY_MIN_BLOCKS) lossy_kernel(const
     if (in_pkt < P.P && e < P.n) nvalid = (P.n - e >= 8) ? 8 : (int)(P.n - e);
     if constexpr (kDevCheck) {   // debug build: the chunk's range, in the slab and in every replica
       const uint64_t c0 = (uint64_t)k * P.P + (uint64_t)c * kChunk;
-      const uint64_t cl = c0 < P.n ? (P.n - c0 < (uint64_t)kChunk ? P.n - c0 : (uint64_t)kChunk) : 0;
+      const uint64_t in_packet = P.P - c * kChunk < (uint32_t)kChunk ? P.P - c * kChunk : (uint32_t)kChunk;   // a chunk ends with its packet
+      const uint64_t cl = c0 < P.n ? (P.n - c0 < in_packet ? P.n - c0 : in_packet) : 0;
       if (!tile_ok(P, k, j, c0, cl, kSiteRegister, lane)) continue;
     }
 

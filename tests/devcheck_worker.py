@@ -14,6 +14,7 @@ CASES = [
     # name, W, n, P, p, optimizer, gradient type, replica type, flags, fused, kernel named in a failed check
     ("register", 8, 2048 * 9 + 77, 2048, 0.2, "adam", "bf16", "bf16", L.LOSSY_REGISTER_PATH, True, "register kernel"),
     ("register_elided", 5, 512 * 23 + 9, 512, 0.3, "sgd", "f32", "bf16", L.LOSSY_REGISTER_PATH | SKIP, True, "register kernel"),
+    ("register_packets_shorter_than_a_chunk_elided", 17, 128 * 60, 128, 0.3, "adam", "bf16", "bf16", L.LOSSY_REGISTER_PATH | SKIP, True, "register kernel"),
     ("fused_bulk", 8, 2048 * 11, 2048, 0.1, "adam", "bf16", "bf16", 0, True, "fused bulk-copy pipeline"),
     ("fused_bulk_elided_w17", 17, 4096 * 40, 4096, 0.3, "adam", "bf16", "f32", SKIP, True, "fused bulk-copy pipeline"),
     ("fused_packed", 16, 256 * 64, 256, 0.1, "adam", "bf16", "bf16", L.LOSSY_PACKED_BULK, True, "fused bulk-copy pipeline (packed)"),
