@@ -351,6 +351,13 @@ bool gather_geometry(const lossy_ctx* ctx, bool rd, TmaGeom& G) {
   // bit 2: the mask warp sends the stale pairs' old copies toward L2 tiles ahead (W = 16, p = 0.1: 0.94 -> 0.99;
   // with more than about two stale replicas per sub-packet it loses: W = 12, p = 0.2: 0.86 -> 0.78)
   G.hints = (c.W - 1) * c.p_param < 1.8 ? 4u : 0u;
+  // bit 3: how the wide geometry's two gather warps share a group. Dealing out the workers halves each warp's
+  // ballots and is ahead wherever rows have holes (W = 16, P = 256: +1 / +7 / +1 % at p = 0.1 / 0.2 / 0.3; P = 512,
+  // p = 0.3: +4 %) and with 9-12 or more than 16 workers at any loss (W = 24: +4 % at p = 0, +6 % at 0.1; W = 64,
+  // P = 512: +9 %); where most rows are whole, up to 8 or with 13-16 workers, both warps in one row do better
+  // (W = 16: 0.98-0.99 against 0.91-0.94 up to p = 0.05; W = 8: +1 %). Same-process A/B pairs, repeatable to 0.002.
+  const double whole_rows = pow(1.0 - c.p_grad, (double)G.packets_per_tile);
+  if (whole_rows >= 0.6 && (c.W <= 8u || (c.W >= 13u && c.W <= 16u))) G.hints |= 8u;
   return true;
 }
 

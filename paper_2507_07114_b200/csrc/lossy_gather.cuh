@@ -377,16 +377,25 @@ __global__ void __launch_bounds__(GatherShape<CW, RD>::kThreads, GatherShape<CW,
         }
         // Delivered pieces of this group's workers: a row is copied in chunks of 512 bytes (one warp
         // instruction, 16 bytes per lane), each lane testing the sub-packet its 16 bytes lie in.
-        for (uint32_t u = 0; u < in_group; ++u) {
+        auto copy_row = [&](uint32_t u, uint32_t c_first, uint32_t c_step) {
           const uint32_t rowmask = __ballot_sync(0xFFFFFFFFu, (recv_l >> (g * kGroup + u)) & 1ull) & 0xFFu;
-          if (rowmask == 0u) continue;
+          if (rowmask == 0u) return;
           const unsigned char* src = reinterpret_cast<const unsigned char*>(P.grads[g * kGroup + u]) + e0 * kGB;
           const uint32_t dst = st + u * kRowG;
 #pragma unroll
-          for (uint32_t c = pw; c < kRowG / 512u; c += kNP) {
+          for (uint32_t c = c_first; c < kRowG / 512u; c += c_step) {
             const uint32_t off = c * 512u + (uint32_t)lane * 16u;   // byte within the row
             if ((rowmask >> ((off / kGB) >> lgP)) & 1u) cp_async16(dst + off, src + off);
           }
+        };
+        // Two gather warps deal out either the group's workers (a row of several chunks per warp and turn: half the
+        // ballots) or every row's chunks (both warps in the same row); the host picks (G.hints bit 3 = chunks).
+        // (One gather warp keeps the loop it had: the same copies written as the two-warp form ran 6-14 % slower in
+        // the twin geometry.)
+        if (kNP > 1 && !(G.hints & 8u)) {
+          for (uint32_t u = pw; u < in_group; u += kNP) copy_row(u, 0u, 1u);
+        } else {
+          for (uint32_t u = 0; u < in_group; ++u) copy_row(u, pw, kNP);
         }
         cp_async_arrive(full_bar(s));
       }

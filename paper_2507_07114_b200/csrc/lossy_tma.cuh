@@ -59,7 +59,7 @@ struct TmaGeom {
   uint32_t state_bytes;       // SPLIT builds: one state slot (theta, m, v, wire tile), 128-byte multiple
   uint32_t groups;            // ceil(W / GS)
   uint32_t grad_slots;        // min(W, GS)
-  uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores, bit 2 (gather pipeline): L2 prefetch of stale copies
+  uint32_t hints;             // bit 0: evict-first on bulk loads, bit 1: on bulk stores, bit 2 (gather pipeline): L2 prefetch of stale copies, bit 3 (gather pipeline): the gather warps split a row's chunks, not the workers
   uint32_t packets_per_tile;  // PACKED build: whole small packets per tile (2, 4 or 8), else 1
   uint32_t full_packets;      // PACKED build: complete packets of the bucket
   uint32_t rd_cap;            // gather pipeline, RD builds: 512-byte chunks per scratch buffer
