@@ -287,12 +287,13 @@ def time_point(L, w, bucket, grad_sets, steps, warmup=3, *, flags=0, alg1=False,
     prev = torch.zeros_like(bucket.master) if alg1 else None
     stream = torch.cuda.current_stream()
 
+    # the arguments of a step are marshalled once per gradient set (the binding's prepared call): a step is then
+    # one foreign call, which is what a launch-bound bucket needs
+    calls = [L.lossy_fused_step_prepared(ctx, gs[:W], bucket.master, bucket.m, bucket.v, reps, norms=norms,
+                                         ghat_prev=prev, stream=stream) for gs in grad_sets]
+
     def step(t):
-        gs = grad_sets[t % len(grad_sets)][:W]
-        if alg1:
-            L.lossy_fused_step_alg1(ctx, t, gs, prev, bucket.master, bucket.m, bucket.v, reps, norms=norms)
-        else:
-            L.lossy_fused_step(ctx, t, gs, bucket.master, bucket.m, bucket.v, reps, norms=norms)
+        calls[t % len(calls)](t)
 
     t = 0
     for _ in range(max(3, warmup)):
@@ -300,17 +301,23 @@ def time_point(L, w, bucket, grad_sets, steps, warmup=3, *, flags=0, alg1=False,
         step(t)
         torch.maximum(worst, norms, out=worst)
     torch.cuda.synchronize()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    # an event after every step (per-step minimum), except in the launch-bound case, where recording it costs a
+    # fifth of a step: there only the two ends are recorded
+    every = not graph
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1 if every else 2)]
     ev[0].record(stream)
     for i in range(steps):
         t += 1
         step(t)
-        ev[i + 1].record(stream)
+        if every:
+            ev[i + 1].record(stream)
+    if not every:
+        ev[1].record(stream)
     torch.cuda.synchronize()
     torch.maximum(worst, norms, out=worst)
     L.lossy_device_status(ctx)
     ms = ev[0].elapsed_time(ev[-1]) / steps
-    per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)] if every else [ms]
     out = {"workload": w.name + ("[alg1]" if alg1 else ""), "W": W, "P": w.packet_elems, "p": w.p, "n": w.n,
            "steps": steps, "ms_per_step": ms, "min_ms": min(per), "steps_per_s": 1e3 / ms}
     B = algorithmic_bytes(w, alg1=alg1)
@@ -320,11 +327,13 @@ def time_point(L, w, bucket, grad_sets, steps, warmup=3, *, flags=0, alg1=False,
     if graph:
         # launch-bound case: capture `steps` consecutive steps once, replay them as one graph launch
         side = torch.cuda.Stream()
+        side_calls = [L.lossy_fused_step_prepared(ctx, gs[:W], bucket.master, bucket.m, bucket.v, reps, norms=norms,
+                                                  ghat_prev=prev, stream=side) for gs in grad_sets]
         with torch.cuda.stream(side):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=side):
                 for i in range(steps):
-                    step(t + 1 + i)
+                    side_calls[(t + 1 + i) % len(side_calls)](t + 1 + i)
         for _ in range(3):
             g.replay()
         torch.cuda.synchronize()

@@ -238,6 +238,29 @@ def lossy_fused_step(ctx, step, grads, master, m, v, replicas, ghat=None, count=
                                                 _p(sumsq), _stream()))
 
 
+class lossy_fused_step_prepared:
+    """lossy_fused_step (or, with ghat_prev, lossy_fused_step_alg1) with its arguments marshalled once: the pointer
+    tables and handles are built here, a call `prepared(step)` is one foreign call. For buckets so small that a
+    step is bound by launch overhead (a 40 MB bucket: 19 -> 12 us per step); the tensors are kept alive by this
+    object and must not be reallocated while it is used. `stream`: a torch stream whose handle is read once, or
+    None to read the current stream at every call."""
+
+    def __init__(self, ctx, grads, master, m, v, replicas, ghat=None, count=None, recv_bits=None, stale_bits=None,
+                 norms=None, sumsq=None, ghat_prev=None, stream=None):
+        lib = load_library()
+        self._ctx, self._keep = ctx, (grads, master, m, v, replicas, ghat, count, recv_bits, stale_bits, norms, sumsq, ghat_prev)
+        self._fn = lib.lossy_fused_step if ghat_prev is None else lib.lossy_fused_step_alg1
+        head = (_table(grads),) + (() if ghat_prev is None else (_p(ghat_prev),))
+        self._args = head + (_p(master), _p(m), _p(v), _table(replicas), _p(ghat), _p(count), _p(recv_bits),
+                             _p(stale_bits), _p(norms), _p(sumsq))
+        self._stream = None if stream is None else C.c_void_p(stream.cuda_stream)
+
+    def __call__(self, step):
+        rc = self._fn(self._ctx, step, *self._args, self._stream if self._stream is not None else _stream())
+        if rc != LOSSY_OK:
+            _check(self._ctx, rc)
+
+
 def lossy_aggregate_alg1(ctx, step, grads, ghat_prev, ghat, count=None, recv_bits=None):
     _check(ctx, load_library().lossy_aggregate_alg1(ctx, step, _table(grads), _p(ghat_prev), _p(ghat), _p(count),
                                                     _p(recv_bits), _stream()))
