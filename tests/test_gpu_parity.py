@@ -114,6 +114,8 @@ EDGE = [
     ("packed_drift_warps_w7_f32_replicas", 7, 256 * 90, 256, 0.45, "adam", "bf16", "f32", 0),
     ("packed_drift_warps_w4_wide", 4, 256 * 75 + 100, 256, 0.3, "adam", "bf16", "bf16", SKIP),
     ("packed_drift_warps_w17_elided", 17, 512 * 40, 512, 0.25, "sgd", "bf16", "bf16", L.LOSSY_REPLICA_SKIP_OWNER),
+    # fp32 replicas leave each drift warp a scratch of four chunks for a mean of 13 stale ones: most come from memory directly
+    ("packed_drift_warps_w16_f32_replicas_direct_loads", 16, 256 * 75, 256, 0.45, "adam", "bf16", "f32", 0),
     # mostly whole rows: the two gather warps deal out every row's chunks instead of the workers
     ("packed_gather_chunks_dealt_w16", 16, 256 * 70 + 24, 256, 0.03, "adam", "bf16", "bf16", 0),
     ("packed_gather_chunks_dealt_w7_512_f32_grads", 7, 512 * 37, 512, 0.05, "sgd", "f32", "bf16", 0),
