@@ -342,6 +342,13 @@ bool gather_geometry(const lossy_ctx* ctx, bool rd, TmaGeom& G) {
     if (G.rd_cap + more > most) more = most > G.rd_cap ? most - G.rd_cap : 0u;
     G.rd_cap += more;
     G.state_bytes += more * scratch_unit;
+    // A drift warp's stale chunks of a tile should mostly fit its scratch: what does not fit is loaded directly at
+    // its full latency. Where not even their mean count fits (fp32 replicas, whose wire ring takes the room: a
+    // scratch of 4 chunks for a mean of 9) the compute warps' reads serve better; the caller falls back to them,
+    // unless it was told to use this build (LOSSY_GATHER_PATH: comparison and tests). (W = 16, P = 256, p = 0.3,
+    // bf16: 8 chunks for a mean of 4.5; W = 24: 8 for 6.9.)
+    const double mean = share / 8.0 * row_chunks * c.p_param * (c.W - 1.0) / c.W;
+    if (!(c.flags & LOSSY_GATHER_PATH) && G.rd_cap < mean) return false;
   }
   G.tiles_per_packet = 1;
   const uint64_t tiles = (kfull + G.packets_per_tile - 1) / G.packets_per_tile;
@@ -436,11 +443,20 @@ int run_tma(lossy_ctx* ctx, const Params& P, bool drift, cudaStream_t s, uint32_
     const double pm = c.p_grad > c.p_param ? c.p_grad : c.p_param;
     const bool wide_fits = c.packet_elems * (uint32_t)kMaxSub >= (uint32_t)GatherShape<16>::kTile;
     const double stale = (c.W - 1u) * c.p_param;
-    const bool drift_warps = wide_fits && c.W >= 4u && c.W <= 24u && stale < 7.5 && stale >= 0.2 * ((double)c.W - 8.0);
-    const bool reg_ahead = !(c.flags & LOSSY_GATHER_PATH) && !drift_warps && ((c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15));
+    // (bf16 replicas: with fp32 ones a row has twice the chunks and the wire ring leaves the drift warps little
+    // scratch; the compute warps' reads gave 0.71-0.73 where drift warps gave 0.48-0.59; LOSSY_GATHER_PATH asks
+    // for the drift warps all the same, for tests)
+    const bool drift_warps = wide_fits && c.W >= 4u && c.W <= 24u && stale < 7.5 && stale >= 0.2 * ((double)c.W - 8.0) &&
+                             (c.replica_dtype == LOSSY_BF16 || (c.flags & LOSSY_GATHER_PATH));
+    // (the register kernel's lead at high loss was measured with bf16 replicas; with fp32 ones the compute warps'
+    // reads are ahead at W = 12-16, p = 0.3: 0.71-0.73 against 0.57-0.62)
+    const bool reg_ahead = !(c.flags & LOSSY_GATHER_PATH) && !drift_warps &&
+                           (c.replica_dtype == LOSSY_BF16 ? (c.W >= 12 && pm >= 0.25) || (c.W >= 24 && pm >= 0.15) : c.W >= 24 && pm >= 0.25);
     if (!reg_ahead) {
       int rc = LOSSY_OK;
       if (c.W >= 4u) rc = try_gather<16>(ctx, P, drift, drift_warps, s, blocks, used);
+      if (rc || *used) return rc;
+      if (c.W > kRdTwinMaxWorkers && drift && drift_warps) rc = try_gather<16>(ctx, P, drift, false, s, blocks, used);   // scratch too small
       if (rc || *used) return rc;
       rc = try_gather<8>(ctx, P, drift, c.W <= kRdTwinMaxWorkers, s, blocks, used);
       if (rc || *used) return rc;

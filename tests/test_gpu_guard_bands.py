@@ -39,7 +39,7 @@ CASES = [
     ("packed_128_twin", 30, 128 * 77 + 8, 128, 0.1, "sgd", "f32", "bf16", L.LOSSY_PACKED_BULK),
     ("gather_wide_256", 16, 256 * 45 + 40, 256, 0.1, "adam", "bf16", "bf16", 0),
     ("gather_wide_drift_warps_256", 16, 256 * 45 + 40, 256, 0.3, "adam", "bf16", "bf16", 0),
-    ("gather_wide_drift_warps_quarters_512_f32_replicas", 5, 512 * 27 + 24, 512, 0.3, "adam", "bf16", "f32", 0),
+    ("gather_wide_drift_warps_quarters_512_f32_replicas", 5, 512 * 27 + 24, 512, 0.3, "adam", "bf16", "f32", L.LOSSY_GATHER_PATH),
     ("gather_wide_drift_warps_scratch_overflow", 24, 256 * 83 + 8, 256, 0.3, "sgd", "bf16", "bf16", 0),
     ("gather_twin_128", 20, 128 * 77 + 8, 128, 0.1, "sgd", "f32", "bf16", 0),
     ("gather_twin_few_workers_512", 3, 512 * 23 + 16, 512, 0.4, "adam", "bf16", "f32", 0),

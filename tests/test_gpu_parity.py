@@ -111,11 +111,12 @@ EDGE = [
     ("packed_drift_warps_w12_halves", 12, 256 * 67 + 9, 256, 0.3, "adam", "bf16", "bf16", 0),
     ("packed_drift_warps_w5_quarters_512", 5, 512 * 41, 512, 0.2, "sgd", "f32", "bf16", 0),
     ("packed_drift_warps_w24_scratch_overflow", 24, 256 * 130 + 8, 256, 0.3, "adam", "bf16", "bf16", 0),
-    ("packed_drift_warps_w7_f32_replicas", 7, 256 * 90, 256, 0.45, "adam", "bf16", "f32", 0),
+    ("packed_drift_warps_w7_f32_replicas", 7, 256 * 90, 256, 0.45, "adam", "bf16", "f32", L.LOSSY_GATHER_PATH),
     ("packed_drift_warps_w4_wide", 4, 256 * 75 + 100, 256, 0.3, "adam", "bf16", "bf16", SKIP),
     ("packed_drift_warps_w17_elided", 17, 512 * 40, 512, 0.25, "sgd", "bf16", "bf16", L.LOSSY_REPLICA_SKIP_OWNER),
-    # fp32 replicas leave each drift warp a scratch of four chunks for a mean of 13 stale ones: most come from memory directly
-    ("packed_drift_warps_w16_f32_replicas_direct_loads", 16, 256 * 75, 256, 0.45, "adam", "bf16", "f32", 0),
+    # fp32 replicas (the policy gives them to the compute warps; the flag asks for drift warps) leave each drift warp a
+    # scratch of four chunks for a mean of 13 stale ones: most come from memory directly
+    ("packed_drift_warps_w16_f32_replicas_direct_loads", 16, 256 * 75, 256, 0.45, "adam", "bf16", "f32", L.LOSSY_GATHER_PATH),
     # mostly whole rows: the two gather warps deal out every row's chunks instead of the workers
     ("packed_gather_chunks_dealt_w16", 16, 256 * 70 + 24, 256, 0.03, "adam", "bf16", "bf16", 0),
     ("packed_gather_chunks_dealt_w7_512_f32_grads", 7, 512 * 37, 512, 0.05, "sgd", "f32", "bf16", 0),
