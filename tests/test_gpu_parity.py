@@ -387,3 +387,18 @@ def test_packed_build_many_tiles_per_cta_with_skewed_stale_sets():
         compare_outputs(gpu.outputs(), ref, f"packed skew step {t}")
         compare_state(gpu, orc, f"packed skew step {t}")
     L.lossy_device_status(gpu.ctx)
+
+
+@pytest.mark.parametrize("W,P,p,plan", [
+    (8, 256, 0.3, "gather wide packets/tile=8 stages=3 drift-warps"),
+    (16, 512, 0.05, "gather wide packets/tile=4 stages=3"),
+    (3, 256, 0.3, "gather twin packets/tile=4 stages=4"),
+])
+def test_gather_pipeline_rings_wrap_element_by_element(W, P, p, plan):
+    """Ten tiles and more per CTA (148 CTAs of 2048-element tiles, or 296 of 1024): the mask ring, the wire ring and
+    the stage ring wrap and their phase bits flip, compared with the oracle element by element over the whole bucket
+    (the full-size tests compare sampled slabs)."""
+    n = 2048 * 148 * 10 + P * 3 + 17
+    w = workload.Workload(f"rings_w{W}_P{P}", W, n, P, p, "adam", 3e-4, "bf16", "bf16", 2, seed=21)
+    gpu, _ = run_parity(w, 2)
+    assert L.lossy_describe_plan(gpu.ctx) == plan
